@@ -30,7 +30,7 @@ class ListReport:
 
 def compare_lists(counts: np.ndarray, indices: np.ndarray, lists: Sequence[np.ndarray], S: np.ndarray,
                   forced: np.ndarray, mode: str, k: int = 0, mass: float = 0.0, tag: str = "",
-                  report: ListReport = None) -> ListReport:
+                  report: ListReport = None, mass_rel: float = None) -> ListReport:
     """counts [n_q], indices [n_q, cap] from the CUDA path for one head; lists/S/forced from the
     oracle.  Differences must lie inside the near-cutoff band and keep the count (top-k) or
     change it by at most one at a mass edge."""
@@ -48,7 +48,8 @@ def compare_lists(counts: np.ndarray, indices: np.ndarray, lists: Sequence[np.nd
         if np.any(np.diff(got) <= 0) or (c and (got[0] < 0 or got[-1] >= S.shape[1])):
             rep.bad.append(f"{tag} row {i}: list not ascending/unique/in range")
             continue
-        ex, edge = orc.near_cutoff_exempt(S[i], forced, "mass" if mode == "mass" else "topk", k=k, mass=mass)
+        ex, edge = orc.near_cutoff_exempt(S[i], forced, "mass" if mode == "mass" else "topk", k=k, mass=mass,
+                                          mass_rel=mass_rel)
         diff = np.setxor1d(got, want)
         if not np.all(ex[diff]):
             rep.bad.append(f"{tag} row {i}: blocks {diff[~ex[diff]][:8]} differ outside the cutoff band")

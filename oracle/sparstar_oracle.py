@@ -189,13 +189,16 @@ def dense_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray, tau: float) -> 
 
 # --------------------------------------------------------------------------- acceptance band
 def near_cutoff_exempt(S_row: np.ndarray, forced: np.ndarray, mode: str, k: int = 0,
-                       mass: float = 0.0, rel: float = 1e-5) -> Tuple[np.ndarray, bool]:
+                       mass: float = 0.0, rel: float = 1e-5, mass_rel: float = None) -> Tuple[np.ndarray, bool]:
     """Blocks of one row whose membership may legitimately differ from the
     oracle's list: selectable blocks whose score lies within rel*|c| of the
     cutoff score c (top-k: the k-th best; mass: the r*-th).  In mass mode the
-    second value tells whether the cumulative mass next to the cutoff is within
-    rel*p of p, in which case blocks r*, r*+1 are exempt and the count may
-    differ by one."""
+    second value tells whether the cumulative mass just before or just after
+    the r*-th block is within mass_rel*p of p (mass_rel defaults to rel); then
+    the prefix may end one block earlier or later, so the blocks of ranks r*
+    and r*+1 are exempt and the count may differ by one.  (Rank r*-1 is never
+    exempt on this account: a prefix that stops before it has a mass further
+    from p than the one that stops before r*.)"""
     sel = np.nonzero(~forced)[0]
     ex = np.zeros(S_row.shape[0], dtype=bool)
     if sel.size == 0:
@@ -203,12 +206,13 @@ def near_cutoff_exempt(S_row: np.ndarray, forced: np.ndarray, mode: str, k: int 
     s = S_row[sel]
     mass_edge = False
     if mode == "mass":
+        width = (rel if mass_rel is None else mass_rel) * mass
         r, order, c = mass_prefix_length(s, mass)
         cut = s[order[r - 1]]
         before = c[r - 2] if r >= 2 else 0.0
-        if abs(c[r - 1] - mass) <= rel * mass or abs(before - mass) <= rel * mass:
+        if abs(c[r - 1] - mass) <= width or abs(before - mass) <= width:
             mass_edge = True
-            ex[sel[order[max(r - 2, 0):r + 1]]] = True
+            ex[sel[order[r - 1:r + 1]]] = True
     else:
         if k <= 0:
             return ex, False

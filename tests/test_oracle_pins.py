@@ -295,6 +295,60 @@ def test_near_cutoff_band_helper():
     assert list(np.nonzero(ex)[0]) == [1]
 
 
+def test_near_cutoff_band_mass_branch_hand_built_rows():
+    """Scores ln(8, 4, 2, 1, 1) on the selectable blocks 1..5 (block 0 is kept): masses 1/2, 1/4,
+    1/8, 1/16, 1/16, cumulative 0.5, 0.75, 0.875, 0.9375, 1."""
+    S = np.concatenate([[99.0], np.log([8.0, 4.0, 2.0, 1.0, 1.0])])
+    forced = np.array([True, False, False, False, False, False])
+    ids = lambda ex: list(np.nonzero(ex)[0])
+    # mass just AFTER rank 2 within 1e-5 p of p from above: r* = 2, the prefix may also run to rank 3
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.75 * (1 - 5e-6))
+    assert edge and ids(ex) == [2, 3]
+    # mass just BEFORE rank 3 within 1e-5 p of p from below: r* = 3, the prefix may also stop at rank 2
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.75 * (1 + 5e-6))
+    assert edge and ids(ex) == [3, 4]
+    # neither: only the score band around the cutoff block (rank 3 = block 3) - and nothing of rank r*-1
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.8)
+    assert not edge and ids(ex) == [3]
+    # just outside the edge (2e-5 p away): no edge
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.75 * (1 - 2e-5))
+    assert not edge and ids(ex) == [2]
+    # a narrower mass edge can be asked for
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.75 * (1 - 5e-6), mass_rel=1e-6)
+    assert not edge and ids(ex) == [2]
+    # r* = 1: "before" is the empty prefix (mass 0)
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.5 * (1 - 5e-6))
+    assert edge and ids(ex) == [1, 2]
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.3)
+    assert not edge and ids(ex) == [1]
+    # equal scores at the cutoff (blocks 4 and 5 tie): both are in the score band
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=0.9)
+    assert not edge and ids(ex) == [4, 5]
+    # r* = last rank: rank r*+1 does not exist
+    ex, edge = orc.near_cutoff_exempt(S, forced, "mass", mass=1.0)
+    assert ids(ex) == [4, 5]
+
+
+def test_compare_lists_uses_the_band_and_nothing_wider():
+    from oracle import compare
+    S = np.concatenate([[99.0], np.log([8.0, 4.0, 2.0, 1.0, 1.0])])[None]
+    forced = np.array([True, False, False, False, False, False])
+    p = 0.75 * (1 + 5e-6)                                    # oracle: r* = 3 -> blocks {0,1,2,3}
+    want = [orc.select_mass_row(S[0], forced, p)]
+    assert list(want[0]) == [0, 1, 2, 3]
+    def rep(row):
+        idx = np.zeros((1, 6), dtype=np.int32)
+        idx[0, :len(row)] = row
+        return compare.compare_lists(np.array([len(row)]), idx, want, S, forced, "mass", mass=p)
+    assert rep([0, 1, 2, 3]).exact == 1
+    r = rep([0, 1, 2])                                        # stopped one early at the mass edge: excused
+    assert r.ok and r.excused == 1
+    assert not rep([0, 1]).ok                                 # two early: not excused
+    assert not rep([0, 1, 3]).ok                              # dropped rank 2 (= r*-1): not excused
+    assert not rep([0, 1, 2, 3, 4, 5]).ok                     # two more blocks: count off by two
+    assert not rep([0, 2, 1, 3]).ok                           # not ascending
+
+
 # ----------------------------------------------------------------- attention-mass analysis
 def test_block_mass_rows_sum_to_one_and_uniform_case():
     b = 4
