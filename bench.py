@@ -23,9 +23,9 @@ sys.path.insert(0, ROOT)
 
 METRIC = "sparse_attn_effective_tflops_kept_blocks"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one sparse attn_tc_kernel launch on config c2 with 4 heads
-# (ncu capture summarised in profiles/attn_tc_kernel_c2_4heads.md), per head; only meaningful for c2-shaped runs
-ATTN_DRAM_BYTES_PER_HEAD = (583.650816e6 + 75.049728e6) / 4
+# dram__bytes_read.sum / dram__bytes_write.sum of one sparse attention launch, as taken from the latest ncu capture
+# of the small (few-head) case of config c2: a small data file kept beside the capture's summary
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "attn_tc_kernel_c2_traffic.json")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -35,6 +35,73 @@ def peaks():
         d = json.load(open(path))
         return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
     return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def measured_traffic(workload_name: str, heads: int, batch: int):
+    """DRAM bytes of one sparse attention launch from the recorded ncu capture, scaled by heads (every
+    head streams its own K/V, so the traffic grows in proportion).  None when no capture of this
+    workload shape is on record."""
+    if not workload_name.startswith("c2") or not os.path.exists(TRAFFIC_FILE):
+        return None, None
+    d = json.load(open(TRAFFIC_FILE))
+    per_head = (float(d["dram_bytes_read"]) + float(d["dram_bytes_write"])) / float(d["heads"])
+    return per_head * heads * batch, d.get("source")
+
+
+def dense_library_times(q, k, v, scale, reps=2):
+    """The dense comparison on library kernels (context for the repo's own dense kernel): torch
+    scaled_dot_product_attention per available backend and FlashAttention-2 if importable, on the
+    same tensors in this GPU's memory.  Returns {name: ms}."""
+    import torch
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    try:
+        from torch.nn.attention import SDPBackend, sdpa_kernel
+        import torch.nn.functional as F
+        for name, be in (("sdpa_flash", SDPBackend.FLASH_ATTENTION), ("sdpa_cudnn", SDPBackend.CUDNN_ATTENTION)):
+            try:
+                def run():
+                    with sdpa_kernel([be]):
+                        return F.scaled_dot_product_attention(q, k, v, scale=scale)
+                out[name] = timed(run)
+            except Exception:
+                torch.cuda.synchronize()
+    except Exception:
+        pass
+    try:
+        from flash_attn import flash_attn_func
+        qt, kt, vt = (t.transpose(1, 2) for t in (q, k, v))            # [B, L, H, D] views
+        out["flash_attn2"] = timed(lambda: flash_attn_func(qt, kt, vt, softmax_scale=scale))
+    except Exception:
+        torch.cuda.synchronize()
+    return out
+
+
+def workload_config(w, in_gb: float, sharding: str):
+    """The `config` object of the JSON line: the same keys and values in the CUDA arm and in the
+    reference arm (static facts of the workload only)."""
+    return {"workload": w.name, "L_q": w.L_q, "L_k": w.L_k, "H": w.H, "D": w.D, "block": w.block, "batch": w.B,
+            "select": w.mode, "mass": w.mass, "ratio": w.ratio,
+            "l2": (f"inputs ({in_gb:.2f} GB) exceed L2; no flush between steps" if in_gb > 0.2 else
+                   f"inputs ({in_gb:.2f} GB) fit L2 and are not flushed: a profiling-size run, not a bench value"),
+            "sharding": sharding}
+
+
+def input_gb(w) -> float:
+    esz = 2 if w.dtype == "bf16" else 4
+    return (w.L_q + 2 * w.L_k) * w.D * w.H * w.B * esz / 1e9
 
 
 def kept_flops(w, num, idx) -> float:
@@ -51,10 +118,23 @@ def kept_flops(w, num, idx) -> float:
     return float((4.0 * w.D * keys * qv).sum().item())
 
 
+SHARDING = {"weak": "one same-shaped workload per GPU, no collective",
+            "strong": "the heads of ONE workload split across the GPUs, no collective"}
+
+
 def rank_workload(w0, rank: int):
-    """Rank r runs the same-shaped workload on its own seed (the path has no exchange step)."""
+    """Weak scaling: rank r runs the same-shaped workload on its own seed (the path has no exchange step)."""
     from dataclasses import replace
     return replace(w0, seed=w0.seed + 1000 * rank) if rank else w0
+
+
+def head_shard(H: int, rank: int, world: int):
+    """Strong scaling: heads [h0, h1) of the one workload that rank `rank` of `world` owns.  Heads are
+    independent (scores, selection and attention are per head), so the shards need no exchange.  The
+    ranges tile 0..H-1 in rank order; the first H % world ranks hold one head more."""
+    base, extra = divmod(H, world)
+    h0 = rank * base + min(rank, extra)
+    return h0, h0 + base + (1 if rank < extra else 0)
 
 
 def reduce_over_ranks(times_ms, flops: float, device, dist=None):
@@ -181,11 +261,22 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
-def run_reference(args):
+def resolve_workload(args):
+    """The workload both arms run: the named configuration with the profiling overrides applied."""
+    from dataclasses import replace
     from workloads import get_config
+    w0 = get_config(args.workload)
+    if args.heads:
+        w0 = replace(w0, H=args.heads, name=f"{w0.name}_h{args.heads}")
+    if args.block:
+        w0 = replace(w0, block=args.block, name=f"{w0.name}_b{args.block}")
+    return w0
+
+
+def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    w = get_config(args.workload)
+    w = resolve_workload(args)
     import numpy as np  # noqa: F401  (loads BLAS before counting threads)
     for _ in range(args.warmup):
         oracle_sample(w, n_units=2, heads=(0,))
@@ -198,8 +289,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "L_q": w.L_q, "L_k": w.L_k, "H": w.H, "D": w.D, "block": w.block,
-                       "select": w.mode, "mass": w.mass},
+            "config": workload_config(w, input_gb(w), SHARDING[args.scaling]),
+            "achieved_density": sum(s["tiles_heads"] for s in vals) / (len(vals) * w.n_q * w.n_k),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -395,6 +486,9 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
     ap.add_argument("--block", type=int, default=0, help="override the workload's selection block size (profiling captures)")
     ap.add_argument("--impl", default="sparstar", choices=["sparstar", "reference"])
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = one workload per GPU (default), strong = the heads of one workload split across GPUs")
+    ap.add_argument("--no-library-dense", action="store_true", help="skip the torch SDPA / FlashAttention-2 dense timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -431,14 +525,17 @@ def main():
     from paper_2608_10519_b200.pipeline import SparstarAttention, _MODES
     from workloads import generate, get_config
 
-    w0 = get_config(args.workload)
-    if args.heads:
-        w0 = replace(w0, H=args.heads, name=f"{w0.name}_h{args.heads}")
-    if args.block:
-        w0 = replace(w0, block=args.block, name=f"{w0.name}_b{args.block}")
-    w = rank_workload(w0, rank)
+    w0 = resolve_workload(args)
     dev = torch.device("cuda", local)
-    x = generate(w, dev)
+    if args.scaling == "strong" and world > 1:
+        if w0.H < world:
+            raise SystemExit(f"--scaling strong needs at least one head per GPU ({w0.H} heads, {world} GPUs)")
+        h0, h1 = head_shard(w0.H, rank, world)
+        x = generate(w0, dev, heads=(h0, h1))                 # this rank's heads of the SAME workload
+        w = replace(w0, H=h1 - h0)
+    else:
+        w = rank_workload(w0, rank)
+        x = generate(w, dev)
     q, k, v = x["q"], x["k"], x["v"]
     eng = SparstarAttention(local)
     ctx = eng.ctx
@@ -503,6 +600,9 @@ def main():
 
     # dense comparison on the same GPU (outside the timed steps)
     dense_ms = None
+    dense_lib = {}
+    if not args.no_dense and not args.no_library_dense and rank == 0 and w.dtype == "bf16":
+        dense_lib = dense_library_times(q, k, v, scale)
     if not args.no_dense:
         od = torch.empty_like(q)
         sp.sparstar_attn_fwd(ctx, q, k, v, od, blk, scale)
@@ -549,25 +649,32 @@ def main():
 
     pk = peaks()
     att_tflops = flops / (t_att * 1e-3) / 1e12
+    traffic, traffic_src = measured_traffic(w0.name, H, B)
+    esz = q.element_size()
+    # bytes one launch must move: Q in, O out, each K/V block once per head (all of them is the upper bound)
+    algo_bytes = float((2 * q.numel() + k.numel() + v.numel()) * esz)
+    dense_all = dict(dense_lib)
+    if dense_ms is not None:
+        dense_all["sparstar_attn_fwd"] = dense_ms
+    dense_best = min(dense_all, key=dense_all.get) if dense_all else None
+    wfull = w0
     pool_bytes = (q.numel() + k.numel()) * q.element_size() + (qbar.numel() + kbar.numel()) * 4
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": args.scaling if world > 1 else "weak",
         "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "L_q": w.L_q, "L_k": w.L_k, "H": H, "D": D, "block": blk, "batch": B,
-                   "select": w.mode, "mass": w.mass, "ratio": w.ratio, "achieved_density": density,
-                   "l2": (f"inputs ({in_gb:.2f} GB) exceed L2; no flush between steps" if in_gb > 0.2 else
-                          f"inputs ({in_gb:.2f} GB) fit L2 and are not flushed: a profiling-size run, not a bench value"),
-                   "sharding": "one same-shaped workload per GPU, no collective"},
+        "config": workload_config(wfull, input_gb(w), SHARDING[args.scaling]),
+        "achieved_density": density,
         "gpu_launches": int(launches),
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": "attn_tc_kernel (sparse forward)", "achieved": att_tflops,
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": att_tflops / pk["bf16_tflops"],
                      "frac_of_sustained": att_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["source"],
-                     "traffic": ATTN_DRAM_BYTES_PER_HEAD * H * B if w0.name.startswith("c2") else None,
-                     "traffic_unit": "bytes per launch",
-                     "traffic_source": "ncu capture of the 4-head case scaled by heads (profiles/attn_tc_kernel_c2_4heads.md)",
+                     "traffic": traffic, "traffic_unit": "bytes per launch", "traffic_source": traffic_src,
+                     "algorithmic_bytes": algo_bytes,
+                     "traffic_over_algorithmic": None if traffic is None else traffic / algo_bytes,
                      "ms_per_launch": t_att, "flops_per_launch": flops,
                      # the same launch counted per kept tile (4*D*b^2 each, padding of partial blocks included),
                      # and against the nominal dense bf16 figure of the part (2,250 TFLOP/s, from its data sheet)
@@ -577,7 +684,12 @@ def main():
         "breakdown_ms": {"pool": t_pool, "score_select": t_sel, "sparse_attn": t_att, "dense_attn": dense_ms},
         "pool_gbs": pool_bytes / (t_pool * 1e-3) / 1e9, "pool_frac_of_hbm": pool_bytes / (t_pool * 1e-3) / 1e9 / pk["hbm_gbs"],
         "selection_overhead": (t_pool + t_sel) / t_att,
-        "speedup_vs_dense": None if dense_ms is None else dense_ms / ms_per_step,
+        # the dense comparison: this library's dense kernel and library kernels on the same tensors; the
+        # speed-up is taken against the FASTEST of them
+        "dense_ms": dense_all, "dense_fastest": dense_best,
+        "dense_sdpa_ms": min([v_ for n_, v_ in dense_lib.items() if n_.startswith("sdpa")], default=None),
+        "speedup_vs_dense": None if dense_best is None else dense_all[dense_best] / ms_per_step,
+        "speedup_vs_own_dense_kernel": None if dense_ms is None else dense_ms / ms_per_step,
         "dense_tflops": None if dense_ms is None else 4.0 * D * w.L_q * w.L_k * H * B / (dense_ms * 1e-3) / 1e12,
     }
     if world == 1 and not args.no_cpu_baseline:

@@ -8,10 +8,17 @@
  *   - All data pointers are DEVICE pointers owned by the caller unless a parameter says
  *     "host".  Nothing is retained after the call returns except by the context.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
- *     The four operator calls only enqueue work; they neither allocate device memory nor
- *     synchronise - with one exception: the context keeps a device scratch buffer (the work
- *     order of the sparse attention), and the first sparse call that needs it, or needs it
- *     larger, waits for the device and allocates it.
+ *     The operator calls only enqueue work; they neither allocate device memory nor
+ *     synchronise - with one exception: the context keeps a device scratch buffer (work order
+ *     and union lists of the sparse attention, pre-scores of SPARSTAR_SCORE_TCGEN05), and a call
+ *     that needs more of it than the context holds allocates a larger buffer first (cudaMalloc).
+ *     The outgrown buffer is kept until sparstar_destroy, never freed earlier: work already
+ *     enqueued, and any CUDA graph captured from earlier calls, go on using the address they were
+ *     given.  CUDA graphs: run every call once eagerly (or call sparstar_reserve_scratch) before
+ *     capturing it; a call that would have to grow the scratch while `stream` is capturing
+ *     returns SPARSTAR_ERR_CAPTURE and enqueues nothing.
+ *   - The context's device must be the calling thread's current device for every call that
+ *     takes a context and a stream (SPARSTAR_ERR_INVALID_ARG otherwise).
  *   - The int return value is a sparstar_status decided on the HOST before any launch
  *     (argument, shape, alignment and support checks).  Conditions found on the DEVICE
  *     (list entry out of range, capacity exceeded, a bounded wait that ran out) are
@@ -40,7 +47,8 @@ typedef enum {
   SPARSTAR_ERR_TIMEOUT = 5,      /* device: a bounded wait expired; while it is on record the tensor-core attention
                                     kernel does no work (outputs unspecified) until sparstar_check clears it */
   SPARSTAR_ERR_CUDA = 6,         /* a CUDA runtime/driver call failed */
-  SPARSTAR_ERR_TOO_LARGE = 7     /* the problem exceeds a fixed built-in limit of the entry point */
+  SPARSTAR_ERR_TOO_LARGE = 7,    /* the problem exceeds a fixed built-in limit of the entry point */
+  SPARSTAR_ERR_CAPTURE = 8       /* the context scratch would have to grow while `stream` is capturing */
 } sparstar_status;
 
 typedef enum { SPARSTAR_F32 = 0, SPARSTAR_BF16 = 1 } sparstar_dtype;
@@ -92,6 +100,15 @@ typedef struct {
  *   sparstar_score_impl); with SPARSTAR_SCORE_TCGEN05 the pre-scores go to `scores_out` when
  *   given, else to the context's scratch buffer (allocated on first use).
  * sparstar_launch_count returns how many kernels this context has launched so far.
+ * sparstar_reserve_scratch grows the context scratch to at least `bytes` now (no-op if it is
+ *   that large already), so that later calls - captured ones in particular - need not;
+ *   sparstar_scratch_bytes returns its present size.
+ * sparstar_set_debug (test aid, not for production use): work_order_on = 0 makes the sparse
+ *   tensor-core attention walk the query tiles in index order instead of longest list first;
+ *   drop_stage >= 0 makes its TMA producer arm the barrier of that list position and copy
+ *   nothing, so that the consumer's bounded wait runs out after about a second, the launch ends
+ *   with SPARSTAR_ERR_TIMEOUT on record and unspecified outputs (exercises the bounded waits
+ *   without faulting anything); drop_stage < 0 switches it off.  Defaults: 1, -1.
  * sparstar_set_trace (profiling aid): `buf` = device array of 4 * capacity * 2 int64, or NULL to
  *   switch tracing off.  While set, the first CTA of the tensor-core attention kernel records
  *   (tag, SM clock modulo 2^26) pairs for its four roles (MMA issuer, softmax warpgroup 0,
@@ -104,6 +121,9 @@ int sparstar_set_attn_impl(sparstar_ctx* ctx, int32_t impl);
 int sparstar_set_score_impl(sparstar_ctx* ctx, int32_t impl);
 int64_t sparstar_launch_count(const sparstar_ctx* ctx);
 int sparstar_set_trace(sparstar_ctx* ctx, int64_t* buf, int32_t capacity, int32_t skip);
+int sparstar_set_debug(sparstar_ctx* ctx, int32_t work_order_on, int32_t drop_stage);
+int sparstar_reserve_scratch(sparstar_ctx* ctx, int64_t bytes, void* stream);
+int64_t sparstar_scratch_bytes(const sparstar_ctx* ctx);
 const char* sparstar_status_string(int status);
 
 /* ---- host integer helpers ---------------------------------------------------------------
@@ -240,7 +260,8 @@ int sparstar_retained_mass(sparstar_ctx* ctx, const float* mass, const int32_t* 
  * GPU that loads the library until the process exits).
  *   Same tensors, lists, scale and lse as sparstar_sparse_attn_fwd, with these limits:
  *     bf16, D = 128, block = 128 only (SPARSTAR_ERR_UNSUPPORTED otherwise);
- *     B * H * ceil(L_q / 128) <= 65536 work items, else SPARSTAR_ERR_TOO_LARGE and nothing runs.
+ *     B * H * ceil(L_q / 128) <= 65536 work items and ceil(L_q / 128) <= 51200 query tiles per
+ *     (batch, head), else SPARSTAR_ERR_TOO_LARGE and nothing is enqueued.
  *   status_out  nullable DEVICE pointer to two int32 {status, site}: zeroed by this call
  *     (stream-ordered) and then written by the kernel with the first device-side condition
  *     (bad list entry, expired wait).  If NULL the built-in word is used and cannot be read back.

@@ -20,11 +20,12 @@ F32, BF16 = 0, 1
 SEL_TOPK_RATIO, SEL_TOPK_COUNT, SEL_MASS = 0, 1, 2
 ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05 = 0, 1, 2
 SCORE_FP64, SCORE_TCGEN05 = 0, 1
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_TOO_LARGE = range(8)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_TOO_LARGE, ERR_CAPTURE = range(9)
 
 EXPORTS = (
     "sparstar_create", "sparstar_destroy", "sparstar_check", "sparstar_set_attn_impl", "sparstar_set_score_impl",
-    "sparstar_launch_count", "sparstar_set_trace", "sparstar_status_string", "sparstar_num_blocks", "sparstar_budget",
+    "sparstar_launch_count", "sparstar_set_trace", "sparstar_set_debug", "sparstar_reserve_scratch",
+    "sparstar_scratch_bytes", "sparstar_status_string", "sparstar_num_blocks", "sparstar_budget",
     "sparstar_forced_count", "sparstar_keep_ranges", "sparstar_density_lookup", "sparstar_schedule_preset",
     "sparstar_pool_blocks", "sparstar_pool_blocks_range", "sparstar_score_select",
     "sparstar_sparse_attn_fwd", "sparstar_attn_fwd", "sparstar_sparse_attn_fwd_static",
@@ -76,6 +77,10 @@ def load() -> C.CDLL:
     lib.sparstar_set_attn_impl.argtypes = [vp, i32]
     lib.sparstar_set_score_impl.argtypes = [vp, i32]
     lib.sparstar_set_trace.argtypes = [vp, vp, i32, i32]
+    lib.sparstar_set_debug.argtypes = [vp, i32, i32]
+    lib.sparstar_reserve_scratch.argtypes = [vp, i64, vp]
+    lib.sparstar_scratch_bytes.argtypes = [vp]
+    lib.sparstar_scratch_bytes.restype = i64
     lib.sparstar_launch_count.argtypes = [vp]
     lib.sparstar_launch_count.restype = i64
     lib.sparstar_status_string.argtypes = [C.c_int]
@@ -162,6 +167,20 @@ def sparstar_set_attn_impl(ctx: int, impl: int) -> None:
 
 def sparstar_set_score_impl(ctx: int, impl: int) -> None:
     _raise(load().sparstar_set_score_impl(ctx, int(impl)), "sparstar_set_score_impl")
+
+
+def sparstar_set_debug(ctx: int, work_order_on: bool = True, drop_stage: int = -1) -> None:
+    """Test aid (see the header): work order on/off, and the list position whose copy the TMA
+    producer of the tensor-core attention skips so that a bounded wait runs out (-1 = off)."""
+    _raise(load().sparstar_set_debug(ctx, 1 if work_order_on else 0, int(drop_stage)), "sparstar_set_debug")
+
+
+def sparstar_reserve_scratch(ctx: int, nbytes: int, stream=None) -> None:
+    _raise(load().sparstar_reserve_scratch(ctx, int(nbytes), _stream(stream)), "sparstar_reserve_scratch")
+
+
+def sparstar_scratch_bytes(ctx: int) -> int:
+    return int(load().sparstar_scratch_bytes(ctx))
 
 
 def sparstar_launch_count(ctx: int) -> int:

@@ -1,6 +1,8 @@
 // C ABI entry points: argument validation, host integer work (block partition, forced block
-// sets of Eq. 3-4, budget of Eq. 5) and dispatch to the kernels.  No entry point below
-// allocates device memory or synchronises except create/destroy/check.
+// sets of Eq. 3-4, budget of Eq. 5) and dispatch to the kernels.  create / destroy / check
+// allocate, free and synchronise; the operator calls only enqueue work, except that a call whose
+// scratch need exceeds what the context holds allocates a larger buffer first (ensure_scratch;
+// sparstar_reserve_scratch does it ahead of time).
 #include <math.h>
 #include <new>
 
@@ -88,19 +90,37 @@ int dispatch_attn(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
 
 }  // namespace
 
-int ensure_scratch(sparstar_ctx* ctx, size_t bytes) {
+int ensure_scratch(sparstar_ctx* ctx, size_t bytes, cudaStream_t s) {
   if (bytes <= ctx->scratch_bytes) return SPARSTAR_OK;
-  // growing frees the old buffer: earlier work that still reads it must have been ordered
-  // before this call on the same stream, so wait for the device once (first use only)
-  SPARSTAR_CUDA_TRY(cudaDeviceSynchronize());
-  if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
-  ctx->scratch = nullptr;
-  ctx->scratch_bytes = 0;
-  const size_t want = bytes < (1u << 20) ? (1u << 20) : bytes;
-  SPARSTAR_CUDA_TRY(cudaMalloc(&ctx->scratch, want));
+  // A stream that is capturing cannot allocate, and a graph captured earlier keeps the address it
+  // was given: the old buffer is therefore never freed before sparstar_destroy, only retired.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  SPARSTAR_CUDA_TRY(cudaStreamIsCapturing(s, &cap));
+  if (cap != cudaStreamCaptureStatusNone) return SPARSTAR_ERR_CAPTURE;
+  if (ctx->scratch != nullptr && ctx->n_retired >= 32) return SPARSTAR_ERR_TOO_LARGE;
+  size_t want = bytes < (1u << 20) ? (1u << 20) : bytes;
+  if (want < ctx->scratch_bytes + ctx->scratch_bytes / 2) want = ctx->scratch_bytes + ctx->scratch_bytes / 2;
+  void* fresh = nullptr;
+  SPARSTAR_CUDA_TRY(cudaMalloc(&fresh, want));
+  if (ctx->scratch != nullptr) ctx->retired[ctx->n_retired++] = ctx->scratch;
+  ctx->scratch = fresh;
   ctx->scratch_bytes = want;
   return SPARSTAR_OK;
 }
+
+int ctx_device_current(const sparstar_ctx* ctx) {
+  int dev = -1;
+  SPARSTAR_CUDA_TRY(cudaGetDevice(&dev));
+  return dev == ctx->device ? SPARSTAR_OK : SPARSTAR_ERR_INVALID_ARG;
+}
+
+// Every operator call: a context, and its device current on the calling thread.
+#define SPARSTAR_CTX_TRY(ctx)                                   \
+  do {                                                          \
+    if ((ctx) == nullptr) return SPARSTAR_ERR_INVALID_ARG;      \
+    const int st__ = ctx_device_current(ctx);                   \
+    if (st__ != SPARSTAR_OK) return st__;                       \
+  } while (0)
 
 extern "C" {
 
@@ -120,6 +140,9 @@ int sparstar_create(sparstar_ctx** out, int device) {
   c->trace = nullptr;
   c->scratch = nullptr;
   c->scratch_bytes = 0;
+  c->n_retired = 0;
+  c->debug_work_order = 1;
+  c->debug_drop_stage = -1;
   c->trace_cap = 0;
   c->trace_skip = 0;
   c->h_status = nullptr;
@@ -142,13 +165,14 @@ int sparstar_destroy(sparstar_ctx* ctx) {
   if (ctx == nullptr) return SPARSTAR_ERR_INVALID_ARG;
   cudaFree(ctx->d_status);
   if (ctx->scratch != nullptr) cudaFree(ctx->scratch);
+  for (int i = 0; i < ctx->n_retired; ++i) cudaFree(ctx->retired[i]);
   cudaFreeHost(ctx->h_status);
   delete ctx;
   return SPARSTAR_OK;
 }
 
 int sparstar_check(sparstar_ctx* ctx, void* stream, int32_t* site) {
-  if (ctx == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   SPARSTAR_CUDA_TRY(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(sparstar_devstatus),
                                     cudaMemcpyDeviceToHost, s));
@@ -179,6 +203,21 @@ int sparstar_set_trace(sparstar_ctx* ctx, int64_t* buf, int32_t capacity, int32_
   return SPARSTAR_OK;
 }
 
+int sparstar_set_debug(sparstar_ctx* ctx, int32_t work_order_on, int32_t drop_stage) {
+  if (ctx == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  ctx->debug_work_order = work_order_on != 0 ? 1 : 0;
+  ctx->debug_drop_stage = drop_stage < 0 ? -1 : drop_stage;
+  return SPARSTAR_OK;
+}
+
+int sparstar_reserve_scratch(sparstar_ctx* ctx, int64_t bytes, void* stream) {
+  SPARSTAR_CTX_TRY(ctx);
+  if (bytes < 0) return SPARSTAR_ERR_INVALID_ARG;
+  return ensure_scratch(ctx, (size_t)bytes, static_cast<cudaStream_t>(stream));
+}
+
+int64_t sparstar_scratch_bytes(const sparstar_ctx* ctx) { return ctx == nullptr ? -1 : (int64_t)ctx->scratch_bytes; }
+
 int64_t sparstar_launch_count(const sparstar_ctx* ctx) { return ctx == nullptr ? -1 : ctx->launches; }
 
 const char* sparstar_status_string(int status) {
@@ -191,6 +230,7 @@ const char* sparstar_status_string(int status) {
     case SPARSTAR_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case SPARSTAR_ERR_CUDA: return "CUDA call failed";
     case SPARSTAR_ERR_TOO_LARGE: return "problem exceeds a fixed built-in limit of this entry point";
+    case SPARSTAR_ERR_CAPTURE: return "the context scratch would have to grow while the stream is capturing";
     default: return "unknown status";
   }
 }
@@ -218,7 +258,8 @@ int32_t sparstar_forced_count(int64_t L_k, int32_t block, const sparstar_range* 
 
 int sparstar_pool_blocks(sparstar_ctx* ctx, const sparstar_tensor* x, int32_t block, float* pooled,
                          void* stream) {
-  if (ctx == nullptr || pooled == nullptr || block <= 0) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (pooled == nullptr || block <= 0) return SPARSTAR_ERR_INVALID_ARG;
   int st = check_tensor(x);
   if (st != SPARSTAR_OK) return st;
   if (!aligned16(pooled)) return SPARSTAR_ERR_INVALID_ARG;
@@ -228,7 +269,8 @@ int sparstar_pool_blocks(sparstar_ctx* ctx, const sparstar_tensor* x, int32_t bl
 
 int sparstar_pool_blocks_range(sparstar_ctx* ctx, const sparstar_tensor* x, int32_t block, int32_t first_block,
                                int32_t n_blocks, float* pooled, void* stream) {
-  if (ctx == nullptr || pooled == nullptr || block <= 0) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (pooled == nullptr || block <= 0) return SPARSTAR_ERR_INVALID_ARG;
   int st = check_tensor(x);
   if (st != SPARSTAR_OK) return st;
   if (!aligned16(pooled)) return SPARSTAR_ERR_INVALID_ARG;
@@ -304,7 +346,8 @@ int sparstar_score_select(sparstar_ctx* ctx, const float* q_pooled, const float*
                           int64_t L_k, double scale, const sparstar_select_params* params,
                           int32_t* kv_num_blocks, int32_t* kv_indices, int32_t cap, float* scores_out,
                           void* stream) {
-  if (ctx == nullptr || q_pooled == nullptr || k_pooled == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (q_pooled == nullptr || k_pooled == nullptr) return SPARSTAR_ERR_INVALID_ARG;
   if (!aligned16(q_pooled) || !aligned16(k_pooled)) return SPARSTAR_ERR_INVALID_ARG;
   SelectArgs a;
   int st = fill_select_args(&a, B, H, n_q, n_k, D, block, L_k, params, kv_num_blocks, kv_indices, cap);
@@ -318,7 +361,7 @@ int sparstar_score_select(sparstar_ctx* ctx, const float* q_pooled, const float*
     // with exact re-scoring next to the cutoff
     float* pre = scores_out;
     if (pre == nullptr) {
-      st = ensure_scratch(ctx, sizeof(float) * (size_t)B * H * n_q * n_k);
+      st = ensure_scratch(ctx, sizeof(float) * (size_t)B * H * n_q * n_k, s);
       if (st != SPARSTAR_OK) return st;
       pre = static_cast<float*>(ctx->scratch);
     }
@@ -332,7 +375,8 @@ int sparstar_score_select(sparstar_ctx* ctx, const float* q_pooled, const float*
 int sparstar_select_from_scores(sparstar_ctx* ctx, const float* scores, int32_t B, int32_t H, int32_t n_q,
                                 int32_t n_k, int32_t block, int64_t L_k, const sparstar_select_params* params,
                                 int32_t* kv_num_blocks, int32_t* kv_indices, int32_t cap, void* stream) {
-  if (ctx == nullptr || scores == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (scores == nullptr) return SPARSTAR_ERR_INVALID_ARG;
   SelectArgs a;
   int st = fill_select_args(&a, B, H, n_q, n_k, 4, block, L_k, params, kv_num_blocks, kv_indices, cap);
   if (st != SPARSTAR_OK) return st;
@@ -344,7 +388,8 @@ int sparstar_select_from_scores(sparstar_ctx* ctx, const float* scores, int32_t 
 
 int sparstar_block_mass(sparstar_ctx* ctx, const sparstar_tensor* q, const sparstar_tensor* k, int32_t block,
                         float scale, const float* lse_dense, float* mass_out, void* stream) {
-  if (ctx == nullptr || lse_dense == nullptr || mass_out == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (lse_dense == nullptr || mass_out == nullptr) return SPARSTAR_ERR_INVALID_ARG;
   int st;
   if ((st = check_tensor(q)) || (st = check_tensor(k))) return st;
   if (k->B != q->B || k->H != q->H || k->D != q->D || k->dtype != q->dtype) return SPARSTAR_ERR_INVALID_ARG;
@@ -356,7 +401,8 @@ int sparstar_block_mass(sparstar_ctx* ctx, const sparstar_tensor* q, const spars
 int sparstar_retained_mass(sparstar_ctx* ctx, const float* mass, const int32_t* kv_num_blocks,
                            const int32_t* kv_indices, int32_t rows, int32_t n_k, int32_t cap, float* out,
                            void* stream) {
-  if (ctx == nullptr || mass == nullptr || kv_num_blocks == nullptr || kv_indices == nullptr || out == nullptr ||
+  SPARSTAR_CTX_TRY(ctx);
+  if (mass == nullptr || kv_num_blocks == nullptr || kv_indices == nullptr || out == nullptr ||
       rows <= 0 || n_k <= 0 || cap <= 0)
     return SPARSTAR_ERR_INVALID_ARG;
   return launch_retained_mass(ctx, mass, kv_num_blocks, kv_indices, rows, n_k, cap, out,
@@ -367,8 +413,8 @@ int sparstar_sparse_attn_fwd(sparstar_ctx* ctx, const sparstar_tensor* q, const 
                              const sparstar_tensor* v, const sparstar_tensor* o, int32_t block,
                              float scale, const int32_t* kv_num_blocks, const int32_t* kv_indices,
                              int32_t cap, float* lse, void* stream) {
-  if (ctx == nullptr || kv_num_blocks == nullptr || kv_indices == nullptr || cap <= 0)
-    return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
+  if (kv_num_blocks == nullptr || kv_indices == nullptr || cap <= 0) return SPARSTAR_ERR_INVALID_ARG;
   int st = check_attn(q, k, v, o, block);
   if (st != SPARSTAR_OK) return st;
   AttnArgs a;
@@ -381,7 +427,7 @@ int sparstar_sparse_attn_fwd(sparstar_ctx* ctx, const sparstar_tensor* q, const 
 int sparstar_attn_fwd(sparstar_ctx* ctx, const sparstar_tensor* q, const sparstar_tensor* k,
                       const sparstar_tensor* v, const sparstar_tensor* o, int32_t block, float scale,
                       float* lse, void* stream) {
-  if (ctx == nullptr) return SPARSTAR_ERR_INVALID_ARG;
+  SPARSTAR_CTX_TRY(ctx);
   int st = check_attn(q, k, v, o, block);
   if (st != SPARSTAR_OK) return st;
   AttnArgs a;

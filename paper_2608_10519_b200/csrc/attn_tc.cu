@@ -37,7 +37,6 @@
 // SPARSTAR_ERR_TIMEOUT, all roles leave their loops, tensor memory is released and the kernel
 // returns.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -151,7 +150,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   volatile uint32_t* trace_smem = reinterpret_cast<volatile uint32_t*>(base_ptr + kOffTrace);
 
   const int h = blockIdx.y, b = blockIdx.z;
-  const int qi = p.order != nullptr ? p.order[((size_t)b * p.H + h) * p.n_q + blockIdx.x] : (int)blockIdx.x;
+  int qi = p.order != nullptr ? p.order[((size_t)b * p.H + h) * p.n_q + blockIdx.x] : (int)blockIdx.x;
+  if (qi < 0 || qi >= p.n_q) {      // a work order that is not this launch's (stale scratch): flag it, stay in bounds
+    if (threadIdx.x == 0) record_status(p.status, SPARSTAR_ERR_BAD_INDEX, -1);
+    qi = (int)blockIdx.x;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t row_id = ((size_t)b * p.H + h) * p.n_qb + qi / p.m;      // the query block's list
   const bool tracing = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0 &&
@@ -797,14 +800,14 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   p.lse_in = nullptr; p.mass_out = nullptr;
   p.order = nullptr;
   const bool want_order = !dense && p.n_q > 1 && (size_t)p.n_q * sizeof(int) <= 200 * 1024 &&
-                          !(getenv("SPARSTAR_TC_ORDER") != nullptr && atoi(getenv("SPARSTAR_TC_ORDER")) == 0);
+                          ctx->debug_work_order != 0;
   // context scratch: [work order: one int per query tile] [union counts] [union lists]
   const size_t tiles = (size_t)a.q.B * a.q.H * p.n_q;
   const size_t order_bytes = (tiles * sizeof(int) + 255) / 256 * 256;
   size_t need = want_order ? order_bytes : 0;
   if (gather > 1) need = 2 * order_bytes + tiles * (size_t)p.n_kb * sizeof(int);
   if (need > 0) {
-    const int st3 = ensure_scratch(ctx, need);
+    const int st3 = ensure_scratch(ctx, need, s);
     if (st3 != SPARSTAR_OK) return st3;
   }
   char* scratch = static_cast<char*>(ctx->scratch);
@@ -840,8 +843,7 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   }
   p.status = ctx->d_status;
   p.trace = ctx->trace; p.trace_cap = ctx->trace_cap; p.trace_skip = ctx->trace_skip;
-  p.debug_drop_stage = -1;
-  if (const char* e = getenv("SPARSTAR_TC_DEBUG_DROP_STAGE")) p.debug_drop_stage = atoi(e);
+  p.debug_drop_stage = ctx->debug_drop_stage;
   dim3 grid(p.n_q, a.q.H, a.q.B);
   int st2;
   if (gather > 1)
@@ -935,6 +937,7 @@ extern "C" int sparstar_sparse_attn_fwd_static(const sparstar_tensor* q, const s
   const int n_q = (q->L + kBlock - 1) / kBlock;
   const long long items = (long long)q->B * q->H * n_q;
   if (items > kStaticOrderItems) return SPARSTAR_ERR_TOO_LARGE;      // the fixed scratch cannot hold the work order
+  if ((size_t)n_q * sizeof(int) > 200 * 1024) return SPARSTAR_ERR_TOO_LARGE;   // the order kernel sorts a head in shared memory
 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int device = 0;
@@ -966,7 +969,6 @@ extern "C" int sparstar_sparse_attn_fwd_static(const sparstar_tensor* q, const s
   p.status = status;
   p.trace = nullptr; p.trace_cap = 0; p.trace_skip = 0;
   p.debug_drop_stage = -1;
-  if ((size_t)n_q * sizeof(int) > 200 * 1024) return SPARSTAR_ERR_TOO_LARGE;
   static bool order_attr[64] = {};
   if (!order_attr[device]) {
     SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));

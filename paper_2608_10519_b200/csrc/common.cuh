@@ -23,6 +23,10 @@ struct sparstar_ctx {
   sparstar_devstatus* h_status;   // pinned host mirror used by sparstar_check
   void* scratch;                  // device scratch owned by the context, grown on first use
   size_t scratch_bytes;
+  void* retired[32];              // outgrown scratch buffers: kept until destroy, because work already
+  int n_retired;                  // enqueued (or a captured graph) may still name their addresses
+  int debug_work_order;           // test switch: 0 = the sparse attention walks query tiles in index order
+  int debug_drop_stage;           // test switch: >= 0 = the TMA producer skips the copy of this list position
   long long* trace;               // optional device buffer for clock stamps (caller-owned)
   int trace_cap;
   int trace_skip;
@@ -52,8 +56,11 @@ __host__ __device__ __forceinline__ bool is_forced(const ForcedBlocks& f, int j)
     if (e__ != cudaSuccess) return SPARSTAR_ERR_CUDA; \
   } while (0)
 
-// Grows the context's device scratch to at least `bytes` (allocates only when it must grow).
-int ensure_scratch(sparstar_ctx* ctx, size_t bytes);
+// Grows the context's device scratch to at least `bytes` (allocates only when it must grow; the
+// outgrown buffer is retired, not freed).  Fails with SPARSTAR_ERR_CAPTURE if `s` is capturing.
+int ensure_scratch(sparstar_ctx* ctx, size_t bytes, cudaStream_t s);
+// SPARSTAR_OK iff the context's device is the calling thread's current device.
+int ctx_device_current(const sparstar_ctx* ctx);
 
 // Launchers implemented in the kernel files; each returns a sparstar_status.
 int launch_pool(sparstar_ctx* ctx, const sparstar_tensor* x, int block, int first_block, int n_blocks, float* pooled,

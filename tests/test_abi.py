@@ -71,3 +71,8 @@ def test_calls_reject_bad_arguments_without_a_gpu(sp):
     assert lib.sparstar_pool_blocks(None, None, 128, None, None) == sp.ERR_INVALID_ARG
     assert lib.sparstar_attn_fwd(None, None, None, None, None, 128, 1.0, None, None) == sp.ERR_INVALID_ARG
     assert lib.sparstar_set_attn_impl(None, 0) == sp.ERR_INVALID_ARG
+    assert lib.sparstar_set_debug(None, 1, -1) == sp.ERR_INVALID_ARG
+    assert lib.sparstar_reserve_scratch(None, 1024, None) == sp.ERR_INVALID_ARG
+    assert lib.sparstar_scratch_bytes(None) == -1
+    assert lib.sparstar_check(None, None, None) == sp.ERR_INVALID_ARG
+    assert "captur" in sp.status_string(sp.ERR_CAPTURE)

@@ -54,69 +54,86 @@ def test_config0_full_parity(eng):
         compare.check_output(f64(od[0, h]), wantd, "f32", f"dense h{h}")
 
 
-def _full_size_case(eng, w, sel_heads, n_hashed, dense_units=2):
-    """Selection on the whole tensor, compared in full on `sel_heads`; sparse attention on the
-    whole tensor in the benchmark's launch configuration with the ORACLE's lists on the sampled
-    heads (the CUDA lists elsewhere), compared on sampled units."""
+ATTN_HEADS = (0, 7, 19, 31)
+
+
+def _full_size_case(eng, w, sel_heads, n_hashed, attn_heads=None, dense_units=0):
+    """Selection on the whole tensor, compared in full on `sel_heads` ("all" = every head); sparse
+    attention on the whole tensor in the benchmark's launch configuration with the ORACLE's lists
+    on those heads (the CUDA lists elsewhere), compared on sampled (head, query block) units of
+    `attn_heads` (default: the selection heads); `dense_units` of those units are also checked
+    on the dense comparison kernel."""
     x = generate(w, "cuda")
     q, k, v = x["q"], x["k"], x["v"]
     num, idx, _ = eng.select(q, k, w.block, w.mode, ratio=w.ratio, mass=w.mass, forced=w.forced_ranges())
     eng.check()
     tau = w.D ** -0.5
+    sel_heads = tuple(range(w.H)) if sel_heads == "all" else tuple(sel_heads)
+    attn_heads = tuple(h for h in (attn_heads or sel_heads) if h in sel_heads)
     rep = compare.ListReport()
+    num_h, idx_h = num[0].cpu().numpy(), idx[0].cpu().numpy()
+    num_o, idx_o = num_h.copy(), idx_h.copy()
     oracle_lists = {}
     for h in sel_heads:
         lists, S, forced = oracle_selection_head(w, q, k, h)
-        oracle_lists[h] = lists
+        if h in attn_heads:
+            oracle_lists[h] = lists
         kk = orc.budget(int((~forced).sum()), w.ratio) if w.mode != "mass" else 0
-        compare.compare_lists(num[0, h].cpu().numpy(), idx[0, h].cpu().numpy(), lists, S, forced, w.mode,
+        compare.compare_lists(num_h[h], idx_h[h], lists, S, forced, w.mode,
                               k=kk, mass=w.mass, tag=f"{w.name} h{h}", report=rep)
         # forced blocks present, rows sorted and unique
         f_ids = np.nonzero(forced)[0]
-        ih, nh = idx[0, h].cpu().numpy(), num[0, h].cpu().numpy()
         for i in range(0, w.n_q, max(1, w.n_q // 50)):
-            row = ih[i, :nh[i]]
+            row = idx_h[h, i, :num_h[h, i]]
             assert np.all(np.diff(row) > 0) and set(f_ids) <= set(row)
+        for i, l in enumerate(lists):                      # outputs are judged with the oracle's lists
+            num_o[h, i] = len(l)
+            idx_o[h, i, :len(l)] = l
+    print(f"{w.name}: lists on {len(sel_heads)} heads: rows {rep.rows} exact {rep.exact} excused {rep.excused}")
     assert rep.ok, rep.bad[:5]
     assert rep.excused <= max(2, rep.rows // 500), (rep.excused, rep.rows)
-    # outputs are judged with the oracle's lists
-    num2, idx2 = num.clone(), idx.clone()
-    for h, lists in oracle_lists.items():
-        for i, l in enumerate(lists):
-            num2[0, h, i] = len(l)
-            idx2[0, h, i, :len(l)] = torch.from_numpy(l).cuda()
+    num2, idx2 = torch.from_numpy(num_o)[None].cuda(), torch.from_numpy(idx_o)[None].cuda()
     o, lse = eng.sparse_forward(q, k, v, w.block, num2, idx2, want_lse=True)
     eng.check()
-    units = [(h, i) for (h, i) in sample_units(w.n_q, w.H, w.seed, n_hashed, heads=tuple(sel_heads))]
-    kcache = {h: (f64(k[0, h]), f64(v[0, h])) for h in sel_heads}
+    units = [(h, i) for (h, i) in sample_units(w.n_q, w.H, w.seed, n_hashed, heads=attn_heads)]
+    kcache = {h: (f64(k[0, h]), f64(v[0, h])) for h in attn_heads}
+    worst = [0.0, 0.0]
     for (h, i) in units:
         r0, r1 = i * w.block, min((i + 1) * w.block, w.L_q)
         Kh, Vh = kcache[h]
         want, want_lse = orc.attention_block(f64(q[0, h, r0:r1]), Kh, Vh, oracle_lists[h][i], w.block, tau)
         compare.check_output(f64(o[0, h, r0:r1]), want, "bf16", f"{w.name} sparse unit h{h} i{i}")
+        mx, mean = compare.output_errors(f64(o[0, h, r0:r1]), want)
+        worst = [max(worst[0], mx), max(worst[1], mean)]
         assert np.abs(f64(lse[0, h, r0:r1]) - want_lse).max() <= 1e-3
+    print(f"{w.name}: sparse attention on {len(units)} units: worst max-abs {worst[0]:.2e}, worst mean-abs {worst[1]:.2e}")
+    if dense_units:
+        del o, lse
+        od = eng.dense_forward(q, k, v, w.block)
+        eng.check()
+        step = max(1, len(units) // dense_units)
+        for (h, i) in units[::step][:dense_units]:
+            r0, r1 = i * w.block, min((i + 1) * w.block, w.L_q)
+            want, _ = orc.dense_attention(f64(q[0, h, r0:r1]), *kcache[h], tau)
+            compare.check_output(f64(od[0, h, r0:r1]), want, "bf16", f"{w.name} dense unit h{h} i{i}")
+        print(f"{w.name}: dense attention checked on {min(dense_units, len(units[::step]))} units")
     return q, k, v, kcache, units, rep
 
 
 def test_config1_mid_scale(eng):
-    w = get_config("c1")
-    q, k, v, kcache, units, rep = _full_size_case(eng, w, sel_heads=(0, 19), n_hashed=3)
-    # dense comparison kernel on the same tensors, two sampled units
-    od = eng.dense_forward(q, k, v, w.block)
-    eng.check()
-    for (h, i) in units[:2]:
-        r0, r1 = i * w.block, min((i + 1) * w.block, w.L_q)
-        want, _ = orc.dense_attention(f64(q[0, h, r0:r1]), *kcache[h], w.D ** -0.5)
-        compare.check_output(f64(od[0, h, r0:r1]), want, "bf16", f"c1 dense unit h{h} i{i}")
+    _full_size_case(eng, get_config("c1"), sel_heads="all", n_hashed=11, attn_heads=ATTN_HEADS, dense_units=2)
 
 
 def test_config2_final_scale(eng):
-    _full_size_case(eng, get_config("c2"), sel_heads=(0, 31), n_hashed=5)
+    """The headline configuration: lists on all 32 heads, sparse attention on 64 (head, query
+    block) units, the dense comparison kernel (the denominator of the speed-up) on 8 of them."""
+    _full_size_case(eng, get_config("c2"), sel_heads="all", n_hashed=11, attn_heads=ATTN_HEADS, dense_units=8)
 
 
 def test_config3_first_clip(eng):
     w = get_config("c3")
-    q, k, v, kcache, units, rep = _full_size_case(eng, w, sel_heads=(7,), n_hashed=5)
+    q, k, v, kcache, units, rep = _full_size_case(eng, w, sel_heads="all", n_hashed=11, attn_heads=ATTN_HEADS,
+                                                  dense_units=8)
     assert rep.exact + rep.excused == rep.rows
 
 
@@ -130,9 +147,10 @@ def test_config3_small_blocks_full_length(eng, block):
 
 
 def test_config4_pyramid_scale(eng):
-    # one scale of the sweep at the extreme densities (cutoff near the median score at 0.5)
-    for d in (0, 4):
-        _full_size_case(eng, pyramid_sweep(d)[1], sel_heads=(3,), n_hashed=2)
+    # one scale of the sweep at the extreme densities (cutoff near the median score at 0.5): the
+    # sparsest on every head, the densest on one
+    _full_size_case(eng, pyramid_sweep(0)[1], sel_heads="all", n_hashed=11, attn_heads=ATTN_HEADS)
+    _full_size_case(eng, pyramid_sweep(4)[1], sel_heads=(3,), n_hashed=2)
 
 
 def test_forward_host_streams_head_chunks(eng):

@@ -500,24 +500,23 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(eng):
     """Failure detection without a fault: the producer is told to arm one stage barrier and copy
     nothing; the MMA role's bounded wait (about a second) runs out, every role leaves its loop,
     tensor memory is released, the kernel returns and the status word says so."""
-    import os
     import paper_2608_10519_b200 as sp
     q = _rand((1, 1, 128, 128), torch.bfloat16, 80)
     k = _rand((1, 1, 128 * 6, 128), torch.bfloat16, 81)
     o = torch.empty_like(q)
-    os.environ["SPARSTAR_TC_DEBUG_DROP_STAGE"] = "1"
+    sp.sparstar_set_debug(eng.ctx, True, 1)
     try:
         sp.sparstar_attn_fwd(eng.ctx, q, k, k, o, 128, 128 ** -0.5)      # one CTA, six tiles
         st, site = sp.sparstar_check(eng.ctx)
     finally:
-        del os.environ["SPARSTAR_TC_DEBUG_DROP_STAGE"]
+        sp.sparstar_set_debug(eng.ctx, True, -1)
     assert st == sp.ERR_TIMEOUT and site != 0
     # several waves of CTAs: once the expiry is on record the remaining CTAs do no work, so the
     # launch ends after about one timeout (one second), not one per wave
     import time
     qw = _rand((1, 1, 128 * 600, 128), torch.bfloat16, 82)
     ow = torch.empty_like(qw)
-    os.environ["SPARSTAR_TC_DEBUG_DROP_STAGE"] = "1"
+    sp.sparstar_set_debug(eng.ctx, True, 1)
     try:
         torch.cuda.synchronize()
         t0 = time.time()
@@ -525,7 +524,7 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(eng):
         st, site = sp.sparstar_check(eng.ctx)
         elapsed = time.time() - t0
     finally:
-        del os.environ["SPARSTAR_TC_DEBUG_DROP_STAGE"]
+        sp.sparstar_set_debug(eng.ctx, True, -1)
     assert st == sp.ERR_TIMEOUT and elapsed < 3.0, elapsed
     # the next call on the same context is healthy
     sp.sparstar_attn_fwd(eng.ctx, q, k, k, o, 128, 128 ** -0.5)
@@ -642,3 +641,71 @@ def test_size_limits_are_reported(eng):
     x = _rand((1, 1, 64, 12), torch.bfloat16, 92)
     with pytest.raises((sp.SparstarError, AssertionError)) as e:
         eng.pool(x, 16)
+
+
+def _random_lists(n_q, n_k, H, seed):
+    rng = np.random.default_rng(seed)
+    return [[np.sort(rng.choice(n_k, size=int(rng.integers(1, n_k + 1)), replace=False)).astype(np.int32)
+             for _ in range(n_q)] for _ in range(H)]
+
+
+def test_scratch_growth_keeps_a_captured_graph_valid():
+    """A graph captured from a sparse call names the context's scratch (the work order).  A later,
+    larger eager call makes the scratch grow; the outgrown buffer must stay alive, so the replay
+    still gives the eager result.  A call that would have to grow the scratch DURING capture is
+    refused with ERR_CAPTURE and enqueues nothing."""
+    import paper_2608_10519_b200 as sp
+    from paper_2608_10519_b200.pipeline import SparstarAttention
+    e = SparstarAttention(0)
+    try:
+        H, L_q, L_k = 2, 128 * 5 + 9, 128 * 12 + 70
+        q, k, v = (_rand((1, H, L, 128), torch.bfloat16, 700 + i) for i, L in enumerate((L_q, L_k, L_k)))
+        num, idx = lists_to_tensors(_random_lists(6, 13, H, 1), 13, "cuda")
+        o = torch.empty_like(q)
+        # no scratch yet: growth inside a capture is refused
+        g0 = torch.cuda.CUDAGraph()
+        status = []
+        with torch.cuda.graph(g0):
+            try:
+                sp.sparstar_sparse_attn_fwd(e.ctx, q, k, v, o, 128, 128 ** -0.5, num, idx)
+            except sp.SparstarError as err:
+                status.append(err.status)
+        assert status == [sp.ERR_CAPTURE] and sp.sparstar_scratch_bytes(e.ctx) == 0
+        # reserve (or run once eagerly), then capture
+        sp.sparstar_reserve_scratch(e.ctx, 1 << 20)
+        small = sp.sparstar_scratch_bytes(e.ctx)
+        assert small >= 1 << 20
+        sp.sparstar_sparse_attn_fwd(e.ctx, q, k, v, o, 128, 128 ** -0.5, num, idx)
+        e.check()
+        want = o.clone()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            sp.sparstar_sparse_attn_fwd(e.ctx, q, k, v, o, 128, 128 ** -0.5, num, idx)
+        # a much larger eager call: the work order of 2 x 4,100 query tiles of 64-token blocks plus
+        # its union lists needs more than the reserved megabyte
+        Lq2, Lk2 = 64 * 8200, 64 * 40
+        q2, k2 = _rand((1, 2, Lq2, 128), torch.bfloat16, 710), _rand((1, 2, Lk2, 128), torch.bfloat16, 711)
+        num2 = torch.full((1, 2, 8200), 2, dtype=torch.int32, device="cuda")
+        idx2 = torch.zeros((1, 2, 8200, 4), dtype=torch.int32, device="cuda")
+        idx2[..., 1] = 7
+        sp.sparstar_sparse_attn_fwd(e.ctx, q2, k2, k2, torch.empty_like(q2), 64, 128 ** -0.5, num2, idx2)
+        e.check()
+        assert sp.sparstar_scratch_bytes(e.ctx) > small
+        o.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        e.check()
+        assert torch.equal(o, want)
+    finally:
+        e.close()
+
+
+def test_context_checks_the_current_device(eng):
+    """Every operator call verifies that the context's device is current (one GPU is visible here,
+    so only the matching case can run; a mismatch returns ERR_INVALID_ARG before any launch)."""
+    import paper_2608_10519_b200 as sp
+    assert torch.cuda.current_device() == 0
+    x = _rand((1, 1, 256, 128), torch.bfloat16, 95)
+    out = eng.pool(x, 128)
+    eng.check()
+    assert out.shape == (1, 1, 2, 128)

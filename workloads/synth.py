@@ -19,7 +19,7 @@ backbone):
 from __future__ import annotations
 
 import math
-from typing import Dict, Tuple
+from typing import Dict, Optional, Tuple
 
 import torch
 
@@ -95,12 +95,18 @@ def _segment_stream(w: Workload, tensor: str, kind: str) -> int:
     return _stream_key(w.seed, _TENSOR_ID[tensor], _KIND_ID[kind], tag)
 
 
-def generate(w: Workload, device="cpu") -> Dict[str, torch.Tensor]:
+def generate(w: Workload, device="cpu", heads: Optional[Tuple[int, int]] = None) -> Dict[str, torch.Tensor]:
     """Returns q [B,H,L_q,D], k, v [B,H,L_k,D] in the workload's dtype on
-    `device` (contiguous)."""
+    `device` (contiguous).  `heads` = (h0, h1) generates only heads h0..h1-1 of
+    the workload (tensors of h1-h0 heads holding exactly the bits those heads
+    have in the full tensors): a rank of a head-sharded run makes its own shard."""
     dt = torch.float32 if w.dtype == "f32" else torch.bfloat16
     dev = torch.device(device)
-    B, H, D = w.B, w.H, w.D
+    B, D = w.B, w.D
+    h0, h1 = (0, w.H) if heads is None else (int(heads[0]), int(heads[1]))
+    if not (0 <= h0 < h1 <= w.H):
+        raise ValueError(f"head range {heads} outside 0..{w.H}")
+    H = h1 - h0
     n_cells = w.cells[0] * w.cells[1]
     q = torch.empty((B, H, w.L_q, D), dtype=dt, device=dev)
     k = torch.empty((B, H, w.L_k, D), dtype=dt, device=dev)
@@ -109,7 +115,7 @@ def generate(w: Workload, device="cpu") -> Dict[str, torch.Tensor]:
     q_cells = _cells(w.q_grid, w.cells, dev)
     for b in range(B):
         for h in range(H):
-            bh = b * H + h
+            bh = b * w.H + h0 + h
             mu = w.alpha * normal_pairs(mu_key, bh * n_cells * D // 2, n_cells * D // 2, dev).reshape(n_cells, D)
             # queries: the current-scale tokens
             L = w.L_q
