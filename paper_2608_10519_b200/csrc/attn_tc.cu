@@ -15,7 +15,7 @@
 //   warps 0-3  softmax warpgroup of stream 0: thread r owns query row r (TMEM lane r)
 //   warps 4-7  softmax warpgroup of stream 1
 //   warp  8    TMA producer
-//   warp  9    MMA issuer: "service u" = O += P_u V_u (P read from tensor memory, where the
+//   warp  9    MMA issuer (whole warp converged, one elected lane issues): "service u" = O += P_u V_u (P read from tensor memory, where the
 //              softmax warpgroup wrote it as bf16 over S) followed at once by S = Q K_{u+2}^T
 //              into the same columns; the tensor pipe runs its instructions in order, so the
 //              overwrite of P_u needs no wait
@@ -314,7 +314,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   } else if (warp == 9) {
     // ================================ MMA issuer ========================================
     reg_dec<kRegsOther>();
-    if (lane == 0 && n > 0) {
+    // All 32 lanes run this loop converged (every value in it is warp-uniform); the MMA and commit
+    // wrappers elect the one lane that issues.  Waits are made warp-uniform with a vote so that no
+    // lane can leave the loop alone.
+    auto wait_all = [&](uint32_t b, uint32_t parity, int site) {
+      return __all_sync(0xffffffffu, mbar_wait(b, parity, abort_flag, site));
+    };
+    if (n > 0) {
       constexpr uint32_t idesc_qk = instr_desc(false, 128u);         // S: 128 queries x 128 keys
       constexpr uint32_t idesc_pv = instr_desc(true, (uint32_t)HD);  // O: 128 queries x HD
       const uint64_t qdesc0 = smem_desc(base + kOffQ, 16, 1024);
@@ -331,7 +337,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           umma_ss(ts, qdesc0 + off, kd + off, idesc_qk, kk > 0 ? 1u : 0u);
         }
       };
-      bool ok = mbar_wait(bar(BAR_Q), 0, abort_flag, 200);
+      bool ok = wait_all(bar(BAR_Q), 0, 200);
       if (ok) {
         tc_fence_after();
         TRACE(0, 20, 0);
@@ -342,7 +348,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           umma_commit(bar(BAR_SFULL + 1));
         }
         TRACE(0, 21, 0);
-        if (!kMass || n > 2) ok = mbar_wait(bar(BAR_STAGE + 0), 0u, abort_flag, 210);
+        if (!kMass || n > 2) ok = wait_all(bar(BAR_STAGE + 0), 0u, 210);
       }
       int st = 0;
       uint32_t sph = 0;
@@ -351,7 +357,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)st * (kTileBytes >> 4));
         const uint32_t to = tO[x], tp = tS[x];
         const uint32_t acc0 = u >= 2 ? 1u : 0u;
-        ok = mbar_wait(bar(BAR_PFULL + x), (uint32_t)(u >> 1) & 1u, abort_flag, 220 + x);
+        ok = wait_all(bar(BAR_PFULL + x), (uint32_t)(u >> 1) & 1u, 220 + x);
         if (!ok) break;
         tc_fence_after();
         TRACE(0, 22, u);
@@ -370,7 +376,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         TRACE(0, 24, u);
         if (++st == kStages) { st = 0; sph ^= 1u; }
         if (kMass ? (u + 3 < n) : (u + 1 < n)) {     // operands of the next service, while this one runs
-          ok = mbar_wait(bar(BAR_STAGE + st), sph, abort_flag, 210 + st);
+          ok = wait_all(bar(BAR_STAGE + st), sph, 210 + st);
           tc_fence_after();
           TRACE(0, 25, u);
         }

@@ -104,7 +104,7 @@ score_tc_kernel(const ScoreTcParams p) {
   tc_fence_after();
   const uint32_t tmem = tmem_slot;
 
-  if (tid == 0) {
+  if (tid < 32) {                                          // warp 0, converged: one elected lane issues
     constexpr uint32_t idesc = instr_desc(false, 128u);
     // (A term, B term) pairs, largest weight first
     const int pa[6] = {0, 0, 1, 1, 0, 2};
