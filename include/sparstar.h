@@ -62,7 +62,10 @@ typedef enum {
 typedef enum {
   SPARSTAR_ATTN_AUTO = 0,        /* tensor-core kernel when the shape allows, else SIMT */
   SPARSTAR_ATTN_SIMT = 1,        /* fp32 FFMA kernel (any supported shape) */
-  SPARSTAR_ATTN_TCGEN05 = 2      /* tcgen05/TMEM/TMA kernel (bf16, D in {64,128}, block in {32,64,128,256,512}) */
+  SPARSTAR_ATTN_TCGEN05 = 2,     /* tcgen05/TMEM/TMA kernels (bf16, D in {64,128}, block in {32,64,128,256,512});
+                                    blocks >= 128 and dense: three score tiles in flight, one accumulator */
+  SPARSTAR_ATTN_TCGEN05_2STREAM = 3  /* same shapes; blocks >= 128 and dense on the older two-stream kernel (two
+                                    score tiles, two accumulators merged at the end) - kept as a cross-check */
 } sparstar_attn_impl;
 
 typedef enum {

@@ -1,0 +1,465 @@
+// Block-sparse / dense attention forward for bf16 on the sm_100a tensor cores, three-tile pipeline
+// (Eq. 7: softmax over the keys of the retained blocks A_i, tiles outside A_i skipped).  Head
+// dimension 128 or 64; selection blocks of 128, 256 or 512 tokens walked as tiles of 128 tokens.
+//
+// One CTA per (batch, head, 128-row query tile).  Tensor memory holds THREE score tiles and ONE
+// output accumulator (S0 | S1 | S2 | O): tile t of the key-block list lives in score buffer t % 3
+// and its softmax is done by warpgroup t % 2, so at any time two tiles are being exponentiated
+// (two warps per scheduler keep the exponential pipe full) while the tensor pipe works on a third.
+// P V products accumulate in list order into the one accumulator; nothing is merged at the end.
+//
+// Roles (384 threads; registers are moved from the third warpgroup to the softmax ones):
+//   warps 0-3  softmax warpgroup 0 (tiles 0, 2, ...): thread r owns query row r (TMEM lane r)
+//   warps 4-7  softmax warpgroup 1 (tiles 1, 3, ...)
+//   warp  8    TMA producer (one lane)
+//   warp  9    MMA issuer (whole warp converged, one elected lane issues)
+//              "service u" = O += P_u V_u (P read from tensor memory, where the softmax wrote it as
+//              bf16 over S) followed at once by S[u % 3] = Q K_{u+3}^T into the same columns (the
+//              tensor pipe runs in order, so the overwrite of P_u needs no wait), then ONE commit
+// Barriers:
+//   STAGE[s]  {V_u, K_{u+3}} landed in slot s = u % 3 (transaction bytes)
+//   SFULL[s]  phase 0 = prologue Q K_s^T complete; phase k >= 1 = service 3(k-1)+s complete.
+//             "S of tile t is ready" = phase t/3 of SFULL[t%3]; "service u is complete" = phase
+//             u/3 + 1 of SFULL[u%3]; the producer refills stage u after phase u/3 of SFULL[u%3]
+//   PFULL[s]  the four warps that own the tile in buffer s have written P (one arrival per warp)
+//
+// Softmax reference.  One accumulator means one reference per query row, shared by the row's two
+// threads (one per warpgroup) through a word in shared memory.  Scaling a row's P, O and
+// denominator by a common power of two changes nothing in floating point, so the reference only
+// has to keep the numbers away from overflow: it is the row maximum of the first tile and is raised
+// only when a tile's exponentials leave the safe range.  The common tile therefore has no row
+// maximum and no hand-over of references: exponentials against the thread's cached reference, one
+// comparison on their sum, and, before P is released, a look at the shared word after the tile
+// before (the other warpgroup's) has been released - the release of tile t-1 is the point at which
+// its owner has decided whether it raised the reference.  If the word differs from the cached
+// value, or the sum is out of range, or the row has no reference yet, the warp takes the slow
+// path: adopt the published reference, take the tile's row maximum, raise the reference if needed
+// (wait until every earlier P V has landed, scale O in place, publish), and redo the tile's P from
+// the scores (lower half still in registers, upper half still in tensor memory).
+//
+// Every wait on an mbarrier is bounded (about a second); on expiry the CTA records
+// SPARSTAR_ERR_TIMEOUT, all roles leave their loops, tensor memory is released and the kernel
+// returns.
+#include "attn_tc.cuh"
+
+namespace {
+
+enum {
+  B3_Q = 0,                 // Q and the first (up to three) K tiles
+  B3_STAGE = 1,             // 3
+  B3_SFULL = B3_STAGE + 3,  // 3
+  B3_PFULL = B3_SFULL + 3,  // 3
+  B3_COUNT = B3_PFULL + 3
+};
+constexpr float kRaiseLog2 = 52.5f;   // a tile whose row maximum exceeds the reference by more than 2^52.5 raises it
+                                      // (128 exponentials of at most 2^53 sum to at most kSumLimit = 2^60)
+
+constexpr uint32_t smem3_tiles(int hd) { return (1u + 2u * kStages) * (128u * (uint32_t)hd * 2u); }
+constexpr uint32_t kOff3Misc = 8u * 16u;                         // after the barrier area (16 slots)
+constexpr uint32_t kOff3Lsum = kOff3Misc + 16u;                  // 2 x 128 floats: partial denominators at the final reference
+constexpr uint32_t kOff3Mref = kOff3Lsum + 2u * 128u * 4u;       // 128 floats: the rows' published references
+constexpr uint32_t kOff3Trace = kOff3Mref + 128u * 4u;
+constexpr uint32_t kTail3Bytes = kOff3Trace + 4u * kTraceSlots * 4u;
+constexpr uint32_t smem3_bytes(int hd) { return smem3_tiles(hd) + kTail3Bytes; }
+static_assert(B3_COUNT <= 16, "barrier area");
+static_assert(smem3_bytes(128) <= 232448u, "shared memory per CTA");
+
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, const TcParams p) {
+  static_assert(HD == 64 || HD == 128, "head dimension");
+  constexpr uint32_t kTileBytes = 128u * HD * 2u;
+  constexpr uint32_t kOffK = kOffQ + kTileBytes;
+  constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
+  constexpr uint32_t kOffTail = kOffV + kStages * kTileBytes;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* tail = smem_raw + kOffTail;
+  if ((base & 1023u) != 0u) {       // swizzled tiles need 1024-byte alignment (uniform exit)
+    if (threadIdx.x == 0) record_status(p.status, SPARSTAR_ERR_CUDA, 902);
+    return;
+  }
+  const uint32_t bar0 = base + kOffTail;
+  auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + kOff3Misc);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + kOff3Misc + 4);
+  volatile float* lsum = reinterpret_cast<volatile float*>(tail + kOff3Lsum);
+  volatile float* mref = reinterpret_cast<volatile float*>(tail + kOff3Mref);
+  volatile uint32_t* trace_smem = reinterpret_cast<volatile uint32_t*>(tail + kOff3Trace);
+
+  const int h = blockIdx.y, b = blockIdx.z;
+  int qi = p.order != nullptr ? p.order[((size_t)b * p.H + h) * p.n_q + blockIdx.x] : (int)blockIdx.x;
+  if (qi < 0 || qi >= p.n_q) {      // a work order that is not this launch's (stale scratch): flag it, stay in bounds
+    if (threadIdx.x == 0) record_status(p.status, SPARSTAR_ERR_BAD_INDEX, -1);
+    qi = (int)blockIdx.x;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const size_t row_id = ((size_t)b * p.H + h) * p.n_qb + qi / p.m;      // the query block's list
+  const bool tracing = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0 &&
+                       (warp == 0 || warp == 4 || warp >= 8);
+  int trace_n = 0;
+  const bool dense = p.kv_num_blocks == nullptr;
+  const int* list = dense ? nullptr : p.kv_indices + row_id * (size_t)p.cap;
+  const int cnt = dense ? 0 : max(min(p.kv_num_blocks[row_id], p.cap), 0);
+  // tiles to walk: every listed block contributes m tiles, except that the last key block may hold fewer
+  int n = dense ? p.n_k : cnt * p.m;
+  if (!dense && p.m > 1 && cnt > 0 && list[cnt - 1] == p.n_kb - 1) n -= p.m * p.n_kb - p.n_k;
+  const int q_row0 = qi * kBlock;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B3_Q), 1);
+    for (int i = 0; i < 3; ++i) {
+      mbar_init(bar(B3_STAGE + i), 1);
+      mbar_init(bar(B3_SFULL + i), 1);
+      mbar_init(bar(B3_PFULL + i), 4);
+    }
+    // an expired wait already on record (this launch or an earlier one): do no work, so that a
+    // failing launch ends after one timeout instead of one per wave of CTAs
+    *abort_flag = *reinterpret_cast<volatile int*>(&p.status->status) == SPARSTAR_ERR_TIMEOUT ? 1 : 0;
+    if (p.trace != nullptr)
+      for (int i = 0; i < 4 * kTraceSlots; ++i) trace_smem[i] = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (threadIdx.x < 128) mref[threadIdx.x] = -INFINITY;
+  if (warp == 9) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tS[3] = {tmem + 0u, tmem + 128u, tmem + 256u};
+  const uint32_t tO = tmem + 384u;
+  const bool live = *abort_flag == 0;
+  if (!live) n = 0;
+
+  if (warp == 8) {
+    // ================================ TMA producer ======================================
+    reg_dec<kRegsOther>();
+    if (lane == 0 && n > 0) {
+      int prev = -1;
+      auto checked = [&](int j, bool first_of_block) {
+        if (j < 0 || j >= p.n_kb || (first_of_block && j <= prev)) {   // malformed: flag it, stay in bounds
+          record_status(p.status, SPARSTAR_ERR_BAD_INDEX, (int)row_id);
+          j = min(max(j, 0), p.n_kb - 1);
+        }
+        prev = j;
+        return j;
+      };
+      // first token row of key tile t
+      auto block_at = [&](int t) {
+        if (dense) return t * kBlock;
+        const int sub = p.m == 1 ? 0 : t % p.m;
+        const int j = checked(list[p.m == 1 ? t : t / p.m], sub == 0);
+        return min(j * p.m + sub, p.n_k - 1) * kBlock;
+      };
+      auto load_tile = [&](const CUtensorMap* map, uint32_t dst, uint32_t barrier, int row) {
+        tma_load_4d(dst, map, barrier, 0, row, h, b);
+        if (HD == 128) tma_load_4d(dst + kHalfBytes, map, barrier, 64, row, h, b);
+      };
+      // Q with the first three score tiles' keys
+      int jt[3] = {0, 0, 0};
+      const int n_pro = min(n, 3);
+      for (int t = 0; t < n_pro; ++t) jt[t] = block_at(t);
+      mbar_expect_tx(bar(B3_Q), kTileBytes * (uint32_t)(1 + n_pro));
+      load_tile(&map_q, base + kOffQ, bar(B3_Q), q_row0);
+      for (int t = 0; t < n_pro; ++t) load_tile(&map_k, base + kOffK + (uint32_t)t * kTileBytes, bar(B3_Q), jt[t]);
+      // stage u = {V_u, K_{u+3}} into slot u % 3, free once phase u/3 of SFULL[u%3] has completed
+      bool ok = true;
+      int st = 0;
+      uint32_t ph = 0;
+      for (int u = 0; u < n && ok; ++u) {
+        const bool more = u + 3 < n;
+        const int jk = more ? block_at(u + 3) : 0;
+        ok = mbar_wait(bar(B3_SFULL + st), ph, abort_flag, 100 + st);
+        if (!ok) break;
+        TRACE(3, 10, u);
+        if (u == p.debug_drop_stage) {
+          mbar_expect_tx(bar(B3_STAGE + st), kTileBytes);               // bytes that never arrive
+        } else {
+          mbar_expect_tx(bar(B3_STAGE + st), more ? 2u * kTileBytes : kTileBytes);
+          load_tile(&map_v, base + kOffV + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), jt[0]);
+          if (more) load_tile(&map_k, base + kOffK + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), jk);
+        }
+        jt[0] = jt[1]; jt[1] = jt[2]; jt[2] = jk;
+        if (++st == kStages) { st = 0; ph ^= 1u; }
+      }
+    }
+  } else if (warp == 9) {
+    // ================================ MMA issuer ========================================
+    reg_dec<kRegsOther>();
+    // All 32 lanes run this loop converged (every value in it is warp-uniform); the MMA and commit
+    // wrappers elect the one lane that issues.  Waits are made warp-uniform with a vote so that no
+    // lane can leave the loop alone.
+    auto wait_all = [&](uint32_t bb, uint32_t parity, int site) {
+      return __all_sync(0xffffffffu, mbar_wait(bb, parity, abort_flag, site));
+    };
+    if (n > 0) {
+      constexpr uint32_t idesc_qk = instr_desc(false, 128u);         // S: 128 queries x 128 keys
+      constexpr uint32_t idesc_pv = instr_desc(true, (uint32_t)HD);  // O: 128 queries x HD
+      const uint64_t qdesc0 = smem_desc(base + kOffQ, 16, 1024);
+      const uint64_t kdesc0 = smem_desc(base + kOffK, 16, 1024);
+      const uint64_t vdesc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
+      auto issue_qk = [&](int slot) {                       // S[slot] = Q K^T with the K tile in `slot`
+        const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)slot * (kTileBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          // 16 contraction elements = 32 bytes inside the swizzle atom; second half 16 KB on
+          const uint64_t off = (uint64_t)((((uint32_t)kk >> 2) * kHalfBytes + ((uint32_t)kk & 3u) * 32u) >> 4);
+          umma_ss(tS[slot], qdesc0 + off, kd + off, idesc_qk, kk > 0 ? 1u : 0u);
+        }
+      };
+      bool ok = wait_all(bar(B3_Q), 0u, 200);
+      if (ok) {
+        tc_fence_after();
+        TRACE(0, 20, 0);
+        for (int t = 0; t < 3 && t < n; ++t) {
+          issue_qk(t);
+          umma_commit(bar(B3_SFULL + t));
+        }
+        TRACE(0, 21, 0);
+        ok = wait_all(bar(B3_STAGE + 0), 0u, 210);
+        if (ok) ok = wait_all(bar(B3_PFULL + 0), 0u, 220);
+        tc_fence_after();
+      }
+      int st = 0;
+      uint32_t ph = 0;                                       // parity of the current lap over the three buffers
+      for (int u = 0; u < n && ok; ++u) {
+        const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)st * (kTileBytes >> 4));
+        TRACE(0, 22, u);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)                        // 16 keys = 16 rows of 128 B; P advances 8 columns
+          umma_ts(tO, tS[st] + (uint32_t)kk * 8u, vd + (uint64_t)((uint32_t)kk * (2048u >> 4)), idesc_pv,
+                  (kk > 0 || u > 0) ? 1u : 0u);
+        if (u + 3 < n) issue_qk(st);
+        umma_commit(bar(B3_SFULL + st));
+        TRACE(0, 24, u);
+        if (++st == kStages) { st = 0; ph ^= 1u; }
+        if (u + 1 < n) {                                      // operands of the next service, while this one runs
+          ok = wait_all(bar(B3_PFULL + st), ph, 220 + st);
+          if (ok) ok = wait_all(bar(B3_STAGE + st), ph, 210 + st);
+          tc_fence_after();
+          TRACE(0, 25, u);
+        }
+      }
+    }
+  } else if (warp >= 10) {
+    reg_dec<kRegsOther>();                                  // idle warps of the third warpgroup
+  } else {
+    // ================================ softmax warpgroups ================================
+    reg_inc<kRegsSoftmax>();
+    const int w = warp >> 2;                        // owner of tiles w, w + 2, ...
+    const int row = (warp & 3) * 32 + lane;         // query row = TMEM lane
+    const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+    const float c = p.scale * 1.4426950408889634f;  // logits in log2 units
+    // valid key columns of the last tile: lists ascend, so only the final entry can be the partial last key block
+    int last_valid = kBlock;
+    if (n > 0 && (dense || list[cnt - 1] == p.n_kb - 1)) last_valid = p.L_k - (p.n_k - 1) * kBlock;
+    float my_ref = -INFINITY;                       // the reference my P and partial denominator are expressed in
+    float l = 0.f;
+    bool ok = true;
+    int sb = w;                                     // t % 3
+    uint32_t sph = 0;                               // (t / 3) & 1
+    for (int t = w; t < n && ok; t += 2) {
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + sb), sph, abort_flag, 300 + w));
+      if (!ok) break;
+      tc_fence_after();
+      TRACE(1 + w, 30, t);
+      int c0 = 32, c1 = 32, c2 = 32, c3 = 32;       // valid columns of the tile's four 32-column segments
+      if (t == n - 1 && last_valid < kBlock) {
+        c0 = min(max(last_valid, 0), 32); c1 = min(max(last_valid - 32, 0), 32);
+        c2 = min(max(last_valid - 64, 0), 32); c3 = min(max(last_valid - 96, 0), 32);
+      }
+      uint32_t sr[128];
+      tmem_ld32(tS[sb] + lane_off + 0u, sr + 0);
+      tmem_ld32(tS[sb] + lane_off + 32u, sr + 32);
+      tmem_ld32(tS[sb] + lane_off + 64u, sr + 64);
+      tmem_ld32(tS[sb] + lane_off + 96u, sr + 96);
+      tmem_wait_ld();
+      if ((c0 & c1 & c2 & c3) != 32) {                        // some segment is not full: -inf there
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i >= c0) sr[i] = 0xff800000u;
+          if (i >= c1) sr[32 + i] = 0xff800000u;
+          if (i >= c2) sr[64 + i] = 0xff800000u;
+          if (i >= c3) sr[96 + i] = 0xff800000u;
+        }
+      }
+      TRACE(1 + w, 31, t);
+      // exponentials of one half of the tile (64 keys) against my_ref, packed and stored as P over
+      // the first 64 columns of the score buffer (a row that has no reference yet gives zeros)
+      auto exp_half = [&](int cc) {
+        const float nmc = my_ref > -INFINITY ? -(my_ref * c) : 0.f;
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float a0, a1;
+          fma2(a0, a1, __uint_as_float(sr[cc * 64 + 2 * i]), __uint_as_float(sr[cc * 64 + 2 * i + 1]), c, nmc);
+          const float p0 = ex2(a0), p1 = ex2(a1);
+          sum[i & 3] += p0 + p1;
+          pk[i] = pack_bf16(p0, p1);
+        }
+        tmem_st32(tS[sb] + lane_off + 32u * cc, pk);
+        return (sum[0] + sum[1]) + (sum[2] + sum[3]);
+      };
+      float tile_sum = 0.f;
+      const bool fresh = __any_sync(0xffffffffu, my_ref == -INFINITY);
+      if (!fresh) tile_sum = exp_half(0) + exp_half(1);
+      // The tile before this one (the other warpgroup's) has been released, hence decided: its
+      // owner published any raise of the reference before it arrived.
+      float cur = my_ref;
+      if (t > 0) {
+        const int pb = sb == 0 ? 2 : sb - 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_PFULL + pb), sb == 0 ? sph ^ 1u : sph, abort_flag, 330 + w));
+        if (!ok) break;
+        cur = mref[row];
+      }
+      const bool slow = fresh || cur != my_ref || !(tile_sum < kSumLimit);     // the last also catches inf and NaN
+      if (__any_sync(0xffffffffu, slow)) {
+        if (cur != my_ref) {                         // adopt the published reference
+          l *= my_ref > -INFINITY ? ex2((my_ref - cur) * c) : 0.f;
+          my_ref = cur;
+        }
+        // the tile's scores again: lower 64 still in registers, upper 64 from tensor memory (P never covers them)
+        tmem_ld32(tS[sb] + lane_off + 64u, sr + 64);
+        tmem_ld32(tS[sb] + lane_off + 96u, sr + 96);
+        tmem_wait_ld();
+        if ((c2 & c3) != 32) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            if (i >= c2) sr[64 + i] = 0xff800000u;
+            if (i >= c3) sr[96 + i] = 0xff800000u;
+          }
+        }
+        float mxa[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mxa[e] = fmaxf(__uint_as_float(sr[e]), __uint_as_float(sr[8 + e]));
+#pragma unroll
+        for (int i = 16; i < 128; i += 16)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) mxa[e] = max3(mxa[e], __uint_as_float(sr[i + e]), __uint_as_float(sr[i + 8 + e]));
+        const float mx = fmaxf(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], max3(mxa[5], mxa[6], mxa[7])));
+        float ref_new = my_ref;
+        if (my_ref == -INFINITY || (mx - my_ref) * c > kRaiseLog2) ref_new = fmaxf(my_ref, mx);
+        const bool changed = ref_new != my_ref;      // false when both are -inf (no valid key seen yet)
+        if (t > 0 && __any_sync(0xffffffffu, changed)) {
+          // every earlier P V must have landed in O: that is the completion of service t - 1
+          const int pb = sb == 0 ? 2 : sb - 1;
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + pb), (sb == 0 ? sph ^ 1u : sph) ^ 1u, abort_flag, 310 + w));
+          if (!ok) break;
+          tc_fence_after();
+          const float alpha = changed ? (my_ref > -INFINITY ? ex2((my_ref - ref_new) * c) : 0.f) : 1.f;
+          tmem_wait_st();
+#pragma unroll 1
+          for (int cc = 0; cc < HD / 32; ++cc) {
+            uint32_t orr[32];
+            tmem_ld32(tO + lane_off + 32u * cc, orr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
+            tmem_st32(tO + lane_off + 32u * cc, orr);
+          }
+          l *= alpha;
+        }
+        if (changed) mref[row] = ref_new;
+        my_ref = ref_new;
+        tile_sum = exp_half(0) + exp_half(1);
+      }
+      TRACE(1 + w, 32, t);
+      l += tile_sum;
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B3_PFULL + sb));
+      TRACE(1 + w, 33, t);
+      sb += 2;
+      if (sb >= 3) { sb -= 3; sph ^= 1u; }
+    }
+    // ---- normalise and write O --------------------------------------------------------------
+    if (ok && n > 0) {                              // the completion of the last service
+      const int lb = (n - 1) % 3;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), (uint32_t)((n - 1) / 3 + 1) & 1u, abort_flag, 320 + w));
+      tc_fence_after();
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");            // every row's last reference is published
+    const float ref = mref[row];
+    lsum[w * 128 + row] = my_ref > -INFINITY ? l * ex2((my_ref - ref) * c) : 0.f;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const int q_row = q_row0 + row;
+    constexpr int kCols = HD / 2;                   // this warpgroup's half of D
+    constexpr int kChunks = kCols / 32;
+    if (*abort_flag == 0 && n > 0) {
+      const float lt = lsum[row] + lsum[128 + row];
+      const float inv = lt > 0.f ? 1.0f / lt : 0.f;
+      const uint32_t col0 = (uint32_t)w * (uint32_t)kCols;
+      uint32_t oa[kChunks][32];
+#pragma unroll
+      for (int cc = 0; cc < kChunks; ++cc) tmem_ld32(tO + lane_off + col0 + 32u * cc, oa[cc]);
+      tmem_wait_ld();
+      if (q_row < p.L_q) {
+        __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o) + b * p.osB + h * p.osH +
+                            (long long)q_row * p.osL + col0;
+        uint32_t out[kChunks * 16];
+#pragma unroll
+        for (int cc = 0; cc < kChunks; ++cc)
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            out[cc * 16 + i] = pack_bf16(__uint_as_float(oa[cc][2 * i]) * inv, __uint_as_float(oa[cc][2 * i + 1]) * inv);
+        uint4* dst = reinterpret_cast<uint4*>(og);
+#pragma unroll
+        for (int i = 0; i < kChunks * 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+        if (p.lse != nullptr && w == 0)
+          p.lse[((size_t)b * p.H + h) * p.L_q + q_row] = lt > 0.f ? ref * p.scale + logf(lt) : -INFINITY;
+      }
+    } else if (n == 0 && live) {
+      if (q_row < p.L_q) {
+        __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o) + b * p.osB + h * p.osH +
+                            (long long)q_row * p.osL + w * kCols;
+        uint4* dst = reinterpret_cast<uint4*>(og);
+#pragma unroll
+        for (int i = 0; i < HD / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (p.lse != nullptr && w == 0) p.lse[((size_t)b * p.H + h) * p.L_q + q_row] = -INFINITY;
+      }
+    }
+  }
+
+  // ---- teardown -----------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    for (int i = threadIdx.x; i < 4 * kTraceSlots; i += kThreads) {
+      const int role = i / kTraceSlots, k = i % kTraceSlots;
+      if (k < p.trace_cap) {
+        p.trace[(role * p.trace_cap + k) * 2] = trace_smem[i] >> 26;
+        p.trace[(role * p.trace_cap + k) * 2 + 1] = trace_smem[i] & 0x3FFFFFFu;
+      }
+    }
+  if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.status, SPARSTAR_ERR_TIMEOUT, *abort_flag);
+}
+
+template <int HD>
+int launch3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p,
+            dim3 grid, cudaStream_t s) {
+  static bool attr_set[64] = {};
+  if (!attr_set[ctx->device & 63]) {
+    // the in-kernel register re-balancing needs the compiled allocation to be what it assumes
+    cudaFuncAttributes fa;
+    SPARSTAR_CUDA_TRY(cudaFuncGetAttributes(&fa, attn_tc3_kernel<HD>));
+    if (2 * 128 * kRegsSoftmax + 128 * kRegsOther > kThreads * fa.numRegs) return SPARSTAR_ERR_UNSUPPORTED;
+    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_tc3_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)smem3_bytes(HD)));
+    attr_set[ctx->device & 63] = true;
+  }
+  attn_tc3_kernel<HD><<<grid, kThreads, smem3_bytes(HD), s>>>(mq, mk, mv, p);
+  return SPARSTAR_OK;
+}
+
+}  // namespace
+
+int launch_attn_tc3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s) {
+  return head_dim == 64 ? launch3<64>(ctx, mq, mk, mv, p, grid, s) : launch3<128>(ctx, mq, mk, mv, p, grid, s);
+}
