@@ -669,7 +669,7 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks,
         "e2e": e2e,
-        "roofline": {"bound": "tensor", "kernel": "attn_tc_kernel (sparse forward)", "achieved": att_tflops,
+        "roofline": {"bound": "tensor", "kernel": "attn_tc3_kernel (sparse forward)", "achieved": att_tflops,
                      "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": att_tflops / pk["bf16_tflops"],
                      "frac_of_sustained": att_tflops / pk["bf16_tflops_sustained"], "peak_source": pk["source"],
                      "traffic": traffic, "traffic_unit": "bytes per launch", "traffic_source": traffic_src,
