@@ -425,35 +425,26 @@ def run_mass_analysis(args):
     forced = w.forced_ranges()
     mass, _ = eng.block_mass(q, k, v, w.block)
     rows = []
-    g = torch.Generator(device="cuda").manual_seed(0)
+    import paper_2608_10519_b200 as sp
 
-    # comparison selectors of the paper's ablation, expressed as score arrays for select_from_scores
-    # (analysis only; the paper defines none of them precisely, so these are this benchmark's forms)
-    def block_centres(seg_len, grid, n_tokens_before):
-        """normalised (t, h, w) centre of every 128-token block that starts inside a visual segment"""
-        T, Hh, W = grid
-        tok = torch.arange(seg_len, device="cuda")
-        pos = torch.stack(((tok // (Hh * W)) / T, ((tok // W) % Hh) / Hh, (tok % W) / W), dim=1).double()
-        return pos
-
-    cur = w.segments[-1]
-    pos_q = block_centres(cur.length, cur.grid, 0)
-    qc = torch.stack([pos_q[i * w.block:min((i + 1) * w.block, w.L_q)].mean(0) for i in range(w.n_q)])
-    key_pos = torch.full((w.L_k, 3), float("nan"), dtype=torch.float64, device="cuda")
-    off = 0
-    for sgm in w.segments:
-        if sgm.grid is not None:
-            key_pos[off:off + sgm.length] = block_centres(sgm.length, sgm.grid, off)
-        off += sgm.length
-    kc = torch.stack([torch.nan_to_num(key_pos[j * w.block:min((j + 1) * w.block, w.L_k)], nan=0.5).mean(0)
-                      for j in range(w.n_k)])
-    # sliding window: nearer in normalised space-time = higher score (same for every head)
-    window = (-torch.cdist(qc, kc)).float().expand(w.B, w.H, w.n_q, w.n_k).contiguous()
-    # cross-scale reuse: the lists a coarser scale would have chosen, carried over by position: scores
-    # from queries pooled over 4 neighbouring blocks (a stale, lower-resolution pattern)
-    qbar, kbar = eng.pool(q, w.block), eng.pool(k, w.block)
-    coarse = torch.nn.functional.avg_pool1d(qbar[0].transpose(1, 2), 4, stride=4, ceil_mode=True).transpose(1, 2)
-    stale = torch.einsum("hid,hjd->hij", coarse.repeat_interleave(4, dim=1)[:, :w.n_q], kbar[0])[None].contiguous()
+    # comparison selectors of the paper's ablation (the library's own definitions; analysis only): score
+    # arrays from the library's generators, turned into lists by sparstar_select_from_scores
+    q_segs = [(w.segments[-1].length, w.segments[-1].grid)]
+    k_segs = [(sg.length, sg.grid) for sg in w.segments]
+    shape = (w.B, w.H, w.n_q, w.n_k)
+    window = torch.empty(shape, dtype=torch.float32, device="cuda")
+    sp.sparstar_window_scores(eng.ctx, q_segs, k_segs, w.block, window)
+    noise = torch.empty(shape, dtype=torch.float32, device="cuda")
+    sp.sparstar_random_scores(eng.ctx, 0, noise)
+    # cross-scale reuse: the aggregated-QK scores of 4x coarser blocks carried over by nearest block centre
+    cb = 4 * w.block
+    _, _, coarse = eng.select(q, k, cb, "topk_ratio", ratio=0.5, forced=forced, want_scores=True)
+    cq_f, ck_f = sp.sparstar_block_centres(q_segs, w.block), sp.sparstar_block_centres(k_segs, w.block)
+    cq_c, ck_c = sp.sparstar_block_centres(q_segs, cb), sp.sparstar_block_centres(k_segs, cb)
+    q_map = torch.tensor(sp.sparstar_nearest_block_map(cq_f, cq_c), dtype=torch.int32, device="cuda")
+    k_map = torch.tensor(sp.sparstar_nearest_block_map(ck_f, ck_c), dtype=torch.int32, device="cuda")
+    stale = torch.empty(shape, dtype=torch.float32, device="cuda")
+    sp.sparstar_remap_scores(eng.ctx, coarse, q_map, k_map, stale)
     # token-wise top-K upper bound (the paper's reference curve): every sampled query keeps its own best
     # rho * L_k keys; plain torch on a sample of rows, analysis only
     rows_s = torch.linspace(0, w.L_q - 1, 512, device="cuda").long()
@@ -462,9 +453,8 @@ def run_mass_analysis(args):
     del logits
     for rho in (0.05, 0.09375, 0.1875, 0.3, 0.5):
         num_a, idx_a, _ = eng.select(q, k, w.block, "topk_ratio", ratio=rho, forced=forced)
-        noise = torch.rand(mass.shape, generator=g, device="cuda")
         r = {}
-        for name, sc in (("exact_block", mass), ("random", noise), ("sliding_window", window), ("stale_coarse_pattern", stale)):
+        for name, sc in (("exact_block", mass), ("random", noise), ("sliding_window", window), ("reuse_of_coarser_blocks", stale)):
             n_, i_ = eng.select_from_scores(sc, w.block, w.L_k, "topk_ratio", ratio=rho, forced=forced)
             r[name] = float(eng.retained_mass(mass, n_, i_).double().mean())
         r["aggregated_qk"] = float(eng.retained_mass(mass, num_a, idx_a).double().mean())

@@ -253,6 +253,44 @@ int sparstar_retained_mass(sparstar_ctx* ctx, const float* mass, const int32_t* 
                            const int32_t* kv_indices, int32_t rows, int32_t n_k, int32_t cap, float* out,
                            void* stream);
 
+/* ---- comparison selectors (the selection-strategy ablation: sliding window, random blocks,
+ * cross-scale reuse; Table "selection strategies") ------------------------------------------------
+ * The paper names these selectors but defines none of them; the definitions here are this
+ * library's, made for analysis on synthetic inputs.  Each call writes a score array
+ * [B,H,n_q,n_k] fp32 for sparstar_select_from_scores, which applies the same budget (Eq. 5), tie
+ * rule and always-kept blocks (Eq. 3) as the method's own selector.
+ *   sparstar_segment: one run of tokens; T > 0 means a raster (t, h, w) grid with T*H*W == length
+ *     (token u sits at t = u / (H*W), h = (u / W) % H, w = u % W), T == 0 means tokens without a
+ *     position (text), which count as sitting at the centre (1/2, 1/2, 1/2).  At most 8 segments.
+ *   sparstar_block_centres (host): centres [n_blocks*3] of the blocks of `block` tokens over the
+ *     concatenated segments: per coordinate the mean over the block's tokens of index/extent
+ *     (integer index sums, one fp64 division per segment, segment order).  Returns n_blocks
+ *     (also when `centres` is NULL), -1 on invalid arguments.
+ *   sparstar_nearest_block_map (host): map[i] = the coarse block whose centre is nearest to fine
+ *     block i (squared Euclidean distance in fp64, ties to the lower index).  Returns n_fine or -1.
+ *   sparstar_window_scores: score[i][j] = -||centre_q(i) - centre_k(j)||, the same for every
+ *     (batch, head); centres are formed on the device exactly as by sparstar_block_centres, the
+ *     distance in fp64 with separately rounded operations, rounded once to fp32.
+ *   sparstar_random_scores: score = u(seed, linear index over [B,H,n_q,n_k]) in [0, 1):
+ *     z = seed + (index + 1) * 0x9E3779B97F4A7C15; z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9;
+ *     z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^= z >> 31; u = (z >> 40) * 2^-24.
+ *   sparstar_remap_scores: out[b][h][i][j] = coarse[b][h][q_map[i]][k_map[j]]: a coarser scale's
+ *     scores (the scores_out of its sparstar_score_select) reused at a finer scale through
+ *     nearest-position maps.  q_map [n_q], k_map [n_k]: DEVICE int32; an entry out of range is
+ *     clamped and SPARSTAR_ERR_BAD_INDEX recorded. */
+typedef struct { int64_t length; int32_t T, H, W; } sparstar_segment;
+int32_t sparstar_block_centres(const sparstar_segment* segs, int32_t n_segs, int32_t block, double* centres);
+int32_t sparstar_nearest_block_map(const double* fine, int32_t n_fine, const double* coarse, int32_t n_coarse,
+                                   int32_t* map);
+int sparstar_window_scores(sparstar_ctx* ctx, const sparstar_segment* q_segs, int32_t n_q_segs,
+                           const sparstar_segment* k_segs, int32_t n_k_segs, int32_t block, int32_t B, int32_t H,
+                           float* scores_out, void* stream);
+int sparstar_random_scores(sparstar_ctx* ctx, uint64_t seed, int32_t B, int32_t H, int32_t n_q, int32_t n_k,
+                           float* scores_out, void* stream);
+int sparstar_remap_scores(sparstar_ctx* ctx, const float* coarse_scores, int32_t B, int32_t H, int32_t n_qc,
+                          int32_t n_kc, const int32_t* q_map, const int32_t* k_map, int32_t n_q, int32_t n_k,
+                          float* scores_out, void* stream);
+
 /* ---- sparstar_sparse_attn_fwd_static -----------------------------------------------------
  * (The paper has no counterpart for this call; it exists for integration reasons only.)
  * The sparse forward for callers that must not allocate device memory - code running inside a

@@ -30,6 +30,8 @@ EXPORTS = (
     "sparstar_pool_blocks", "sparstar_pool_blocks_range", "sparstar_score_select",
     "sparstar_sparse_attn_fwd", "sparstar_attn_fwd", "sparstar_sparse_attn_fwd_static",
     "sparstar_block_mass", "sparstar_select_from_scores", "sparstar_retained_mass",
+    "sparstar_block_centres", "sparstar_nearest_block_map", "sparstar_window_scores", "sparstar_random_scores",
+    "sparstar_remap_scores",
 )
 
 
@@ -45,6 +47,10 @@ class _Range(C.Structure):
 
 class _DensityEntry(C.Structure):
     _fields_ = [("L_q", C.c_int64), ("rho", C.c_double)]
+
+
+class _Segment(C.Structure):
+    _fields_ = [("length", C.c_int64), ("T", C.c_int32), ("H", C.c_int32), ("W", C.c_int32)]
 
 
 class _Tensor(C.Structure):
@@ -106,6 +112,14 @@ def load() -> C.CDLL:
     lib.sparstar_block_mass.argtypes = [vp, tp, tp, i32, flt, vp, vp, vp]
     lib.sparstar_select_from_scores.argtypes = [vp, vp, i32, i32, i32, i32, i32, i64, C.POINTER(_SelectParams), vp, vp, i32, vp]
     lib.sparstar_retained_mass.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp]
+    sp_ = C.POINTER(_Segment)
+    lib.sparstar_block_centres.argtypes = [sp_, i32, i32, C.POINTER(dbl)]
+    lib.sparstar_block_centres.restype = i32
+    lib.sparstar_nearest_block_map.argtypes = [C.POINTER(dbl), i32, C.POINTER(dbl), i32, C.POINTER(i32)]
+    lib.sparstar_nearest_block_map.restype = i32
+    lib.sparstar_window_scores.argtypes = [vp, sp_, i32, sp_, i32, i32, i32, i32, vp, vp]
+    lib.sparstar_random_scores.argtypes = [vp, C.c_uint64, i32, i32, i32, i32, vp, vp]
+    lib.sparstar_remap_scores.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, i32, i32, vp, vp]
     lib.sparstar_sparse_attn_fwd_static.argtypes = [tp, tp, tp, tp, i32, flt, vp, vp, i32, vp, vp, vp]
     _lib = lib
     return lib
@@ -358,3 +372,62 @@ def sparstar_retained_mass(ctx: int, mass: torch.Tensor, kv_num_blocks: torch.Te
     _raise(load().sparstar_retained_mass(ctx, mass.data_ptr(), kv_num_blocks.data_ptr(), kv_indices.data_ptr(),
                                          B * H * n_q, n_k, kv_indices.shape[3], out.data_ptr(), _stream(stream)),
            "sparstar_retained_mass")
+
+
+# ---- comparison selectors -----------------------------------------------------------------
+def _segments(segs):
+    """segs: sequence of (length, grid) with grid = (T, H, W) or None for tokens without a position."""
+    arr = (_Segment * max(1, len(segs)))()
+    for i, (length, grid) in enumerate(segs):
+        arr[i].length = int(length)
+        arr[i].T, arr[i].H, arr[i].W = (0, 0, 0) if grid is None else tuple(int(x) for x in grid)
+    return arr
+
+
+def sparstar_block_centres(segs, block: int):
+    """Host helper: list of (t, h, w) centres of the blocks over the concatenated segments."""
+    arr = _segments(segs)
+    n = load().sparstar_block_centres(arr, len(segs), int(block), None)
+    if n < 0:
+        raise ValueError("sparstar_block_centres: invalid arguments")
+    out = (C.c_double * (3 * n))()
+    load().sparstar_block_centres(arr, len(segs), int(block), out)
+    return [(out[3 * i], out[3 * i + 1], out[3 * i + 2]) for i in range(n)]
+
+
+def sparstar_nearest_block_map(fine, coarse):
+    """Host helper: for every fine centre the index of the nearest coarse centre (ties: lower index)."""
+    nf, nc = len(fine), len(coarse)
+    f = (C.c_double * (3 * nf))(*[x for c in fine for x in c])
+    c = (C.c_double * (3 * nc))(*[x for cc in coarse for x in cc])
+    out = (C.c_int32 * nf)()
+    if load().sparstar_nearest_block_map(f, nf, c, nc, out) < 0:
+        raise ValueError("sparstar_nearest_block_map: invalid arguments")
+    return list(out)
+
+
+def sparstar_window_scores(ctx: int, q_segs, k_segs, block: int, scores_out: torch.Tensor, stream=None) -> None:
+    B, H = scores_out.shape[:2]
+    assert scores_out.dtype == torch.float32 and scores_out.is_contiguous() and scores_out.is_cuda
+    _raise(load().sparstar_window_scores(ctx, _segments(q_segs), len(q_segs), _segments(k_segs), len(k_segs), int(block),
+                                         B, H, scores_out.data_ptr(), _stream(stream)), "sparstar_window_scores")
+
+
+def sparstar_random_scores(ctx: int, seed: int, scores_out: torch.Tensor, stream=None) -> None:
+    B, H, n_q, n_k = scores_out.shape
+    assert scores_out.dtype == torch.float32 and scores_out.is_contiguous() and scores_out.is_cuda
+    _raise(load().sparstar_random_scores(ctx, int(seed), B, H, n_q, n_k, scores_out.data_ptr(), _stream(stream)),
+           "sparstar_random_scores")
+
+
+def sparstar_remap_scores(ctx: int, coarse_scores: torch.Tensor, q_map: torch.Tensor, k_map: torch.Tensor,
+                          scores_out: torch.Tensor, stream=None) -> None:
+    B, H, n_qc, n_kc = coarse_scores.shape
+    n_q, n_k = scores_out.shape[2:]
+    assert coarse_scores.dtype == torch.float32 and coarse_scores.is_contiguous() and coarse_scores.is_cuda
+    assert scores_out.dtype == torch.float32 and scores_out.is_contiguous() and tuple(scores_out.shape[:2]) == (B, H)
+    assert q_map.dtype == torch.int32 and k_map.dtype == torch.int32 and q_map.is_cuda and k_map.is_cuda
+    assert q_map.is_contiguous() and k_map.is_contiguous() and q_map.numel() == n_q and k_map.numel() == n_k
+    _raise(load().sparstar_remap_scores(ctx, coarse_scores.data_ptr(), B, H, n_qc, n_kc, q_map.data_ptr(),
+                                        k_map.data_ptr(), n_q, n_k, scores_out.data_ptr(), _stream(stream)),
+           "sparstar_remap_scores")

@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsparstar.so")
-SOURCES = ["api.cu", "pool.cu", "score_select.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc3.cu", "score_tc.cu"]
+SOURCES = ["api.cu", "pool.cu", "score_select.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc3.cu", "score_tc.cu", "selectors.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
