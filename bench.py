@@ -324,12 +324,14 @@ def run_pyramid(args):
             pyr.forward(q, k, v)
         torch.cuda.synchronize()
         reps = max(3, args.steps)
+        l0 = sp.sparstar_launch_count(eng.ctx)
         e0, e1 = ev(), ev()
         e0.record()
         for _ in range(reps):
             pyr.forward(q, k, v)
         e1.record()
         torch.cuda.synchronize()
+        launches = (sp.sparstar_launch_count(eng.ctx) - l0) // reps     # fused selection, work order, attention
         t_sparse = e0.elapsed_time(e1) / reps
         eng.dense_forward(q, k, v, w.block)
         torch.cuda.synchronize()
@@ -343,7 +345,8 @@ def run_pyramid(args):
         num, idx = pyr.select(q, k)
         eng.check()
         out.append({"L_q": w.L_q, "L_k": w.L_k, "rho": pyr.density(w.L_q), "kept_density": float(num.double().mean()) / w.n_k,
-                    "sparse_step_ms": t_sparse, "dense_ms": t_dense, "speedup": t_dense / t_sparse})
+                    "sparse_step_ms": t_sparse, "dense_ms": t_dense, "speedup": t_dense / t_sparse,
+                    "launches_per_scale": int(launches)})
         tot_s += t_sparse
         tot_d += t_dense
         del x, q, k, v

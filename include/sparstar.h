@@ -204,6 +204,24 @@ int sparstar_score_select(sparstar_ctx* ctx, const float* q_pooled, const float*
                           int32_t* kv_num_blocks, int32_t* kv_indices, int32_t cap,
                           float* scores_out, void* stream);
 
+/* ---- sparstar_select_fused -----------------------------------------------------------------
+ * Pooling of Q and K, block scores and selection of one scale in ONE launch (the three steps of
+ * Sec. "Aggregated Query-Key Block Selector" before the attention: block means, Eq. 2, Eq. 5-6),
+ * with the lists sparstar_pool_blocks + sparstar_score_select give, bit for bit.
+ *   q [B,H,L_q,D], k [B,H,L_k,D]   as for sparstar_pool_blocks
+ *   k_cond_pooled / n_cond   nullable [B,H,n_cond,D] fp32: block means of the first n_cond key
+ *       blocks, computed earlier (conditioning keys that do not change between the scales of a
+ *       clip, Sec. "Preliminaries"); those blocks are copied, not pooled again.  Only blocks that
+ *       lie wholly inside the unchanged part may be passed.
+ *   q_pooled [B,H,n_q,D], k_pooled [B,H,n_k,D]   fp32 work arrays, written in full
+ *   params, scale, kv_num_blocks, kv_indices, cap   as for sparstar_score_select
+ * A cooperative launch: the grid is as large as the device holds at once and meets at a grid-wide
+ * barrier between pooling and selection. */
+int sparstar_select_fused(sparstar_ctx* ctx, const sparstar_tensor* q, const sparstar_tensor* k, int32_t block,
+                          double scale, const sparstar_select_params* params, const float* k_cond_pooled,
+                          int32_t n_cond, float* q_pooled, float* k_pooled, int32_t* kv_num_blocks,
+                          int32_t* kv_indices, int32_t cap, void* stream);
+
 /* ---- sparstar_sparse_attn_fwd -----------------------------------------------------------
  * O_t = sum_u softmax_u(scale * q_t . k_u) v_u over keys u < L_k whose block pi_k(u) is in
  * A_{pi_q(t)} (Eq. 7; the key tail is the padding mask).  Forward only.

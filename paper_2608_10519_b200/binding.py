@@ -27,7 +27,7 @@ EXPORTS = (
     "sparstar_launch_count", "sparstar_set_trace", "sparstar_set_debug", "sparstar_reserve_scratch",
     "sparstar_scratch_bytes", "sparstar_status_string", "sparstar_num_blocks", "sparstar_budget",
     "sparstar_forced_count", "sparstar_keep_ranges", "sparstar_density_lookup", "sparstar_schedule_preset",
-    "sparstar_pool_blocks", "sparstar_pool_blocks_range", "sparstar_score_select",
+    "sparstar_pool_blocks", "sparstar_pool_blocks_range", "sparstar_score_select", "sparstar_select_fused",
     "sparstar_sparse_attn_fwd", "sparstar_attn_fwd", "sparstar_sparse_attn_fwd_static",
     "sparstar_block_mass", "sparstar_select_from_scores", "sparstar_retained_mass",
     "sparstar_block_centres", "sparstar_nearest_block_map", "sparstar_window_scores", "sparstar_random_scores",
@@ -107,6 +107,7 @@ def load() -> C.CDLL:
     lib.sparstar_schedule_preset.restype = i32
     lib.sparstar_score_select.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i64, dbl,
                                           C.POINTER(_SelectParams), vp, vp, i32, vp, vp]
+    lib.sparstar_select_fused.argtypes = [vp, tp, tp, i32, dbl, C.POINTER(_SelectParams), vp, i32, vp, vp, vp, vp, i32, vp]
     lib.sparstar_sparse_attn_fwd.argtypes = [vp, tp, tp, tp, tp, i32, flt, vp, vp, i32, vp, vp]
     lib.sparstar_attn_fwd.argtypes = [vp, tp, tp, tp, tp, i32, flt, vp, vp]
     lib.sparstar_block_mass.argtypes = [vp, tp, tp, i32, flt, vp, vp, vp]
@@ -293,6 +294,33 @@ def sparstar_score_select(ctx: int, q_pooled: torch.Tensor, k_pooled: torch.Tens
         ctx, q_pooled.data_ptr(), k_pooled.data_ptr(), B, H, n_q, n_k, D, int(block), int(L_k), float(scale),
         C.byref(p), kv_num_blocks.data_ptr(), kv_indices.data_ptr(), cap,
         None if scores_out is None else scores_out.data_ptr(), _stream(stream)), "sparstar_score_select")
+
+
+def sparstar_select_fused(ctx: int, q: torch.Tensor, k: torch.Tensor, block: int, scale: float, mode: int,
+                          q_pooled: torch.Tensor, k_pooled: torch.Tensor, kv_num_blocks: torch.Tensor,
+                          kv_indices: torch.Tensor, ratio: float = 0.0, count: int = 0, mass: float = 0.0,
+                          forced: Sequence[Tuple[int, int]] = (), k_cond_pooled: Optional[torch.Tensor] = None,
+                          stream=None) -> None:
+    """Pooling + scores + selection of one scale in one launch (see the header)."""
+    B, H, L_q, D = q.shape
+    n_q, n_k = sparstar_num_blocks(L_q, block), sparstar_num_blocks(k.shape[2], block)
+    for t, n in ((q_pooled, n_q), (k_pooled, n_k)):
+        assert t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (B, H, n, D)
+    assert kv_num_blocks.dtype == torch.int32 and kv_indices.dtype == torch.int32
+    assert kv_num_blocks.is_contiguous() and kv_indices.is_contiguous()
+    assert tuple(kv_num_blocks.shape) == (B, H, n_q) and tuple(kv_indices.shape[:3]) == (B, H, n_q)
+    n_cond = 0
+    if k_cond_pooled is not None:
+        assert k_cond_pooled.dtype == torch.float32 and k_cond_pooled.is_contiguous()
+        assert tuple(k_cond_pooled.shape[:2]) == (B, H) and k_cond_pooled.shape[3] == D
+        n_cond = k_cond_pooled.shape[2]
+    tq, tk = _tensor(q), _tensor(k)
+    arr = _ranges(forced)
+    p = _SelectParams(int(mode), int(count), float(ratio), float(mass), arr, len(forced))
+    _raise(load().sparstar_select_fused(
+        ctx, C.byref(tq), C.byref(tk), int(block), float(scale), C.byref(p),
+        None if k_cond_pooled is None else k_cond_pooled.data_ptr(), n_cond, q_pooled.data_ptr(), k_pooled.data_ptr(),
+        kv_num_blocks.data_ptr(), kv_indices.data_ptr(), kv_indices.shape[3], _stream(stream)), "sparstar_select_fused")
 
 
 def sparstar_sparse_attn_fwd(ctx: int, q, k, v, o, block: int, scale: float, kv_num_blocks: torch.Tensor,

@@ -372,6 +372,30 @@ int sparstar_score_select(sparstar_ctx* ctx, const float* q_pooled, const float*
   return launch_score_select(ctx, a, s);
 }
 
+int sparstar_select_fused(sparstar_ctx* ctx, const sparstar_tensor* q, const sparstar_tensor* k, int32_t block, double scale,
+                          const sparstar_select_params* params, const float* k_cond_pooled, int32_t n_cond,
+                          float* q_pooled, float* k_pooled, int32_t* kv_num_blocks, int32_t* kv_indices, int32_t cap,
+                          void* stream) {
+  SPARSTAR_CTX_TRY(ctx);
+  if (q_pooled == nullptr || k_pooled == nullptr || block <= 0) return SPARSTAR_ERR_INVALID_ARG;
+  int st;
+  if ((st = check_tensor(q)) || (st = check_tensor(k))) return st;
+  if (k->B != q->B || k->H != q->H || k->D != q->D || k->dtype != q->dtype) return SPARSTAR_ERR_INVALID_ARG;
+  if (!aligned16(q_pooled) || !aligned16(k_pooled)) return SPARSTAR_ERR_INVALID_ARG;
+  if (n_cond < 0 || (n_cond > 0 && (k_cond_pooled == nullptr || !aligned16(k_cond_pooled)))) return SPARSTAR_ERR_INVALID_ARG;
+  const int n_q = (int)((q->L + block - 1) / block), n_k = (int)((k->L + block - 1) / block);
+  // cached means are valid only for blocks that hold no token past the conditioning part; the caller
+  // says how many such blocks it has
+  if (n_cond > n_k) return SPARSTAR_ERR_INVALID_ARG;
+  SelectArgs a;
+  st = fill_select_args(&a, q->B, q->H, n_q, n_k, q->D, block, k->L, params, kv_num_blocks, kv_indices, cap);
+  if (st != SPARSTAR_OK) return st;
+  a.scale = scale;
+  a.scores_out = nullptr;
+  return launch_select_fused(ctx, a, *q, *k, block, n_cond, k_cond_pooled, n_cond, q_pooled, k_pooled,
+                             static_cast<cudaStream_t>(stream));
+}
+
 int sparstar_select_from_scores(sparstar_ctx* ctx, const float* scores, int32_t B, int32_t H, int32_t n_q,
                                 int32_t n_k, int32_t block, int64_t L_k, const sparstar_select_params* params,
                                 int32_t* kv_num_blocks, int32_t* kv_indices, int32_t cap, void* stream) {

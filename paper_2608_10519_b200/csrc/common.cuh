@@ -84,6 +84,9 @@ struct SelectArgs {
   float* scores_out;
 };
 int launch_score_select(sparstar_ctx* ctx, const SelectArgs& a, cudaStream_t s);
+int launch_select_fused(sparstar_ctx* ctx, const SelectArgs& a, const sparstar_tensor& q, const sparstar_tensor& k, int block,
+                        int first_k_block, const float* k_cond_pooled, int n_cond, float* q_pooled, float* k_pooled,
+                        cudaStream_t s);
 bool score_tc_supported(int D, long long BH);
 int launch_score_tc(sparstar_ctx* ctx, const float* q_pooled, const float* k_pooled, int BH, int n_q, int n_k, int D,
                     float scale, float* scores, cudaStream_t s);

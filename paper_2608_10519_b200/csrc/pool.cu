@@ -5,80 +5,18 @@
 // HBM-bound: every input byte is read once with 16-byte loads, coalesced along D (a warp
 // covers whole consecutive rows), fp32 accumulation in a fixed order, one fp32 row written
 // per block.  One CTA per (batch, head, block).
-#include "common.cuh"
+#include "pool.cuh"
 
 namespace {
 
-constexpr int kPoolThreads = 256;
-
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-  static constexpr int N = 4;
-  __device__ static void add(float* acc, const uint4& u) {
-    acc[0] += __uint_as_float(u.x); acc[1] += __uint_as_float(u.y);
-    acc[2] += __uint_as_float(u.z); acc[3] += __uint_as_float(u.w);
-  }
-};
-template <> struct Vec16<__nv_bfloat16> {
-  static constexpr int N = 8;
-  __device__ static void add(float* acc, const uint4& u) {
-    // bf16 -> fp32 is a 16-bit shift
-    acc[0] += __uint_as_float(u.x << 16); acc[1] += __uint_as_float(u.x & 0xffff0000u);
-    acc[2] += __uint_as_float(u.y << 16); acc[3] += __uint_as_float(u.y & 0xffff0000u);
-    acc[4] += __uint_as_float(u.z << 16); acc[5] += __uint_as_float(u.z & 0xffff0000u);
-    acc[6] += __uint_as_float(u.w << 16); acc[7] += __uint_as_float(u.w & 0xffff0000u);
-  }
-};
-
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-
-// vl = 16-byte vectors per row; groups = row groups that fit in the CTA.
 template <typename T>
 __global__ void __launch_bounds__(kPoolThreads, 8)
 pool_kernel(const T* __restrict__ x, float* __restrict__ pooled, int H, int L, int D, int nb,
             long long sB, long long sH, long long sL, int block, int vl, int groups, int first_block) {
-  constexpr int N = Vec16<T>::N;
   extern __shared__ float part[];             // [groups][D]
   const int blk = first_block + blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int lane = threadIdx.x % vl;
-  const int grp = threadIdx.x / vl;
-  const int r0 = blk * block;
-  const int valid = min(block, L - r0);
-  const T* base = x + b * sB + h * sH + (long long)r0 * sL;
-
-  float acc[N];
-#pragma unroll
-  for (int i = 0; i < N; ++i) acc[i] = 0.f;
-  if (grp < groups) {
-    int r = grp;
-    // four independent 16-byte loads in flight per thread
-    for (; r + 3 * groups < valid; r += 4 * groups) {
-      uint4 u0 = ld_stream(reinterpret_cast<const uint4*>(base + (long long)r * sL) + lane);
-      uint4 u1 = ld_stream(reinterpret_cast<const uint4*>(base + (long long)(r + groups) * sL) + lane);
-      uint4 u2 = ld_stream(reinterpret_cast<const uint4*>(base + (long long)(r + 2 * groups) * sL) + lane);
-      uint4 u3 = ld_stream(reinterpret_cast<const uint4*>(base + (long long)(r + 3 * groups) * sL) + lane);
-      Vec16<T>::add(acc, u0); Vec16<T>::add(acc, u1); Vec16<T>::add(acc, u2); Vec16<T>::add(acc, u3);
-    }
-    for (; r < valid; r += groups) {
-      uint4 u = ld_stream(reinterpret_cast<const uint4*>(base + (long long)r * sL) + lane);
-      Vec16<T>::add(acc, u);
-    }
-#pragma unroll
-    for (int i = 0; i < N; ++i) part[grp * D + lane * N + i] = acc[i];
-  }
-  __syncthreads();
-  const float inv = 1.0f / (float)block;
-  float* out = pooled + (((long long)b * H + h) * nb + blk) * D;
-  for (int d = threadIdx.x; d < D; d += kPoolThreads) {
-    float s = 0.f;
-    for (int g = 0; g < groups; ++g) s += part[g * D + d];
-    out[d] = s * inv;
-  }
+  pool_block_body<T>(x + b * sB + h * sH, pooled + (((long long)b * H + h) * nb + blk) * D, L, D, sL, block, vl, groups,
+                     blk, part);
 }
 
 }  // namespace

@@ -9,11 +9,14 @@
 // finds the cutoff by a bitwise search on order-preserving keys (top-k: k-th largest score;
 // mass: largest cutoff whose softmax mass still reaches p), then emits forced and selected
 // blocks in ascending order by ballot compaction - sorted and unique by construction.
-#include "common.cuh"
+#include <cooperative_groups.h>
+
+#include "pool.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
+static_assert(kThreads == kPoolThreads, "the fused kernel runs the pooling routine with the selection kernel's threads");
 constexpr int kWarps = kThreads / 32;
 constexpr int kRegElems = 36;          // rows of up to 32 * 36 = 1,152 key blocks are searched in registers
 
@@ -56,19 +59,25 @@ struct Params {
   int R;          // query blocks per CTA
 };
 
+// Pooled vectors: through the read-only path when an earlier launch wrote them; through L2 when this
+// very kernel wrote them before a grid-wide barrier (the fused kernel), where the read-only path
+// would be allowed to return stale lines.
+template <bool kSameKernel> __device__ __forceinline__ float4 ld_pooled4(const float4* ptr) {
+  return kSameKernel ? __ldcg(ptr) : __ldg(ptr);
+}
+template <bool kSameKernel> __device__ __forceinline__ float ld_pooled(const float* ptr) {
+  return kSameKernel ? __ldcg(ptr) : *ptr;
+}
+
+// The strip of R query blocks starting at i0 of (batch, head) bh: scores, then selection.
 // Shared memory: qd [D][R] double | S [R][n_k] double | E [R][n_k] double (mass mode on approximate scores only)
-template <int R>
-__global__ void __launch_bounds__(kThreads)
-score_select_kernel(const Params p) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+template <int R, bool kSameKernel>
+__device__ __forceinline__ void score_select_body(const Params& p, const int bh, const int i0, unsigned char* smem_raw) {
   const SelectArgs& a = p.a;
   const int D = a.D, n_k = a.n_k, n_q = a.n_q;
   double* qd = reinterpret_cast<double*>(smem_raw);
   double* S = qd + (size_t)D * R;
   double* E = S + (size_t)R * n_k;
-
-  const int bh = blockIdx.y;
-  const int i0 = blockIdx.x * R;
   const int tid = threadIdx.x;
 
   if (a.scores_in != nullptr) {
@@ -82,7 +91,7 @@ score_select_kernel(const Params p) {
   for (int e = tid; e < R * D; e += kThreads) {
     const int r = e / D, d = e % D;
     const int i = i0 + r;
-    qd[d * R + r] = (i < n_q) ? (double)a.q_pooled[((size_t)bh * n_q + i) * D + d] : 0.0;
+    qd[d * R + r] = (i < n_q) ? (double)ld_pooled<kSameKernel>(a.q_pooled + ((size_t)bh * n_q + i) * D + d) : 0.0;
   }
   __syncthreads();
 
@@ -107,7 +116,7 @@ score_select_kernel(const Params p) {
       float4 kv[8];
 #pragma unroll
       for (int s_ = 0; s_ < 8; ++s_)
-        kv[s_] = (s_ < steps && col < n_k) ? __ldg(kp + 4 * s_) : make_float4(0.f, 0.f, 0.f, 0.f);
+        kv[s_] = (s_ < steps && col < n_k) ? ld_pooled4<kSameKernel>(kp + 4 * s_) : make_float4(0.f, 0.f, 0.f, 0.f);
       double c0 = 0.0, c1 = 0.0;
 #pragma unroll
       for (int s_ = 0; s_ < 8; ++s_) {
@@ -141,8 +150,8 @@ score_select_kernel(const Params p) {
     const float4* kp = reinterpret_cast<const float4*>(kb + (size_t)j * D);
     const float4* kp2 = reinterpret_cast<const float4*>(kb + (size_t)(two ? j2 : j) * D);
     for (int d4 = 0; d4 < D / 4; ++d4) {
-      const float4 kv = __ldg(kp + d4);
-      const float4 kw = __ldg(kp2 + d4);
+      const float4 kv = ld_pooled4<kSameKernel>(kp + d4);
+      const float4 kw = ld_pooled4<kSameKernel>(kp2 + d4);
       const double k0 = kv.x, k1 = kv.y, k2 = kv.z, k3 = kv.w;
       const double w0 = kw.x, w1 = kw.y, w2 = kw.z, w3 = kw.w;
       const double* q = qd + (size_t)d4 * 4 * R;
@@ -389,7 +398,7 @@ score_select_kernel(const Params p) {
         if (fabs(key_to_score(((unsigned long long)kk.x << 32) | kk.y) - cut) > delta) continue;
         const float* krow = a.k_pooled + ((size_t)bh * n_k + j) * D;
         double acc = 0.0;
-        for (int d = 0; d < D; ++d) acc = fma((double)qrow[d], (double)krow[d], acc);
+        for (int d = 0; d < D; ++d) acc = fma((double)ld_pooled<kSameKernel>(qrow + d), (double)ld_pooled<kSameKernel>(krow + d), acc);
         const double sx = a.scale * acc;
         const unsigned long long key = order_key(sx);
         Kr[j] = make_uint2((uint32_t)(key >> 32), (uint32_t)key);
@@ -426,6 +435,71 @@ score_select_kernel(const Params p) {
       a.kv_num_blocks[(size_t)bh * n_q + i] = written;
       if (written > a.cap) record_status(p.status, SPARSTAR_ERR_CAPACITY, i);
     }
+  }
+}
+
+template <int R>
+__global__ void __launch_bounds__(kThreads)
+score_select_kernel(const Params p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  score_select_body<R, false>(p, blockIdx.y, blockIdx.x * R, smem_raw);
+}
+
+// Pooling, scores and selection of one scale in ONE launch (cooperative: the grid is resident as a
+// whole and meets at a grid-wide barrier).  Phase A: block means of Q (all blocks) and of K (blocks
+// from first_k_block on; the means of the blocks before it - conditioning keys that do not change
+// between the scales of a clip - are copied from k_cond_pooled), by the pooling kernel's own block
+// routine, hence with its bits.  Phase B: the strips of the selection kernel, taken round-robin.
+struct FusedParams {
+  Params sel;
+  const void* q; const void* k;          // [B,H,L,D] in the dtype T
+  long long q_sB, q_sH, q_sL, k_sB, k_sH, k_sL;
+  int L_q, L_k, block, vl, groups;
+  int first_k_block;                     // K blocks below it come from k_cond_pooled
+  const float* k_cond_pooled;            // [B,H,n_cond,D]
+  int n_cond;
+  float* q_pooled; float* k_pooled;      // written here, read by phase B
+};
+
+template <int R, typename T>
+__global__ void __launch_bounds__(kThreads)
+select_fused_kernel(const FusedParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const SelectArgs& a = p.sel.a;
+  const int BH = a.B * a.H, D = a.D;
+  float* part = reinterpret_cast<float*>(smem_raw);
+  // ---- phase A -----------------------------------------------------------------------------
+  const int kb_new = a.n_k - p.first_k_block;
+  const long long n_items = (long long)BH * (a.n_q + kb_new);
+  for (long long it = blockIdx.x; it < n_items; it += gridDim.x) {
+    const int bh = (int)(it / (a.n_q + kb_new)), r = (int)(it % (a.n_q + kb_new));
+    const int b = bh / a.H, h = bh % a.H;
+    if (r < a.n_q)
+      pool_block_body<T, true>(static_cast<const T*>(p.q) + b * p.q_sB + h * p.q_sH, p.q_pooled + ((size_t)bh * a.n_q + r) * D,
+                         p.L_q, D, p.q_sL, p.block, p.vl, p.groups, r, part);
+    else
+      pool_block_body<T, true>(static_cast<const T*>(p.k) + b * p.k_sB + h * p.k_sH,
+                         p.k_pooled + ((size_t)bh * a.n_k + p.first_k_block + (r - a.n_q)) * D, p.L_k, D, p.k_sL, p.block,
+                         p.vl, p.groups, p.first_k_block + (r - a.n_q), part);
+    __syncthreads();
+  }
+  if (p.first_k_block > 0) {                     // cached means of the conditioning blocks
+    const long long n4 = (long long)BH * p.first_k_block * (D / 4);
+    for (long long e = (long long)blockIdx.x * kThreads + threadIdx.x; e < n4; e += (long long)gridDim.x * kThreads) {
+      const int d4 = (int)(e % (D / 4));
+      const long long row = e / (D / 4);
+      const int bh = (int)(row / p.first_k_block), j = (int)(row % p.first_k_block);
+      reinterpret_cast<float4*>(p.k_pooled + ((size_t)bh * a.n_k + j) * D)[d4] =
+          __ldg(reinterpret_cast<const float4*>(p.k_cond_pooled + ((size_t)bh * p.n_cond + j) * D) + d4);
+    }
+  }
+  __threadfence();
+  cooperative_groups::this_grid().sync();
+  // ---- phase B -----------------------------------------------------------------------------
+  const int strips = (a.n_q + R - 1) / R;
+  for (long long it = blockIdx.x; it < (long long)BH * strips; it += gridDim.x) {
+    score_select_body<R, true>(p.sel, (int)(it / strips), (int)(it % strips) * R, smem_raw);
+    __syncthreads();
   }
 }
 
@@ -490,4 +564,68 @@ int launch_score_select(sparstar_ctx* ctx, const SelectArgs& a, cudaStream_t s) 
   if (smem_bytes(a, 2) <= limit) return launch_R<2>(ctx, a, s);
   if (smem_bytes(a, 1) <= limit) return launch_R<1>(ctx, a, s);
   return SPARSTAR_ERR_UNSUPPORTED;
+}
+
+
+// ---- pooling + scores + selection in one cooperative launch ----------------------------------
+namespace {
+
+template <int R, typename T>
+int launch_fused_RT(sparstar_ctx* ctx, FusedParams& p, size_t smem, cudaStream_t s) {
+  static bool attr_set[64] = {};
+  static int blocks_per_sm[64] = {};
+  static size_t smem_seen[64] = {};
+  const int dev = ctx->device & 63;
+  if (!attr_set[dev]) {
+    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(select_fused_kernel<R, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    attr_set[dev] = true;
+  }
+  if (blocks_per_sm[dev] == 0 || smem_seen[dev] != smem) {
+    int nb = 0;
+    SPARSTAR_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, select_fused_kernel<R, T>, kThreads, smem));
+    if (nb <= 0) return SPARSTAR_ERR_UNSUPPORTED;
+    blocks_per_sm[dev] = nb;
+    smem_seen[dev] = smem;
+  }
+  p.sel.R = R;
+  void* args[] = {&p};
+  SPARSTAR_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)select_fused_kernel<R, T>, dim3(ctx->sm_count * blocks_per_sm[dev]),
+                                                dim3(kThreads), args, smem, s));
+  ctx->launches++;
+  return SPARSTAR_OK;
+}
+
+template <typename T>
+int launch_fused_T(sparstar_ctx* ctx, FusedParams& p, cudaStream_t s) {
+  const SelectArgs& a = p.sel.a;
+  const size_t pool_smem = (size_t)p.groups * a.D * sizeof(float);
+  const size_t limit = 200 * 1024;
+  auto need = [&](int R) { const size_t b = smem_bytes(a, R); return b > pool_smem ? b : pool_smem; };
+  if (need(8) <= limit) return launch_fused_RT<8, T>(ctx, p, need(8), s);
+  if (need(4) <= limit) return launch_fused_RT<4, T>(ctx, p, need(4), s);
+  if (need(2) <= limit) return launch_fused_RT<2, T>(ctx, p, need(2), s);
+  if (need(1) <= limit) return launch_fused_RT<1, T>(ctx, p, need(1), s);
+  return SPARSTAR_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+int launch_select_fused(sparstar_ctx* ctx, const SelectArgs& a, const sparstar_tensor& q, const sparstar_tensor& k, int block,
+                        int first_k_block, const float* k_cond_pooled, int n_cond, float* q_pooled, float* k_pooled,
+                        cudaStream_t s) {
+  if (a.D % 4 != 0 || (long long)a.B * a.H > 65535) return SPARSTAR_ERR_UNSUPPORTED;
+  const int esz = q.dtype == SPARSTAR_BF16 ? 2 : 4;
+  const int row_bytes = q.D * esz;
+  if (row_bytes % 16 != 0 || row_bytes > 4096) return SPARSTAR_ERR_UNSUPPORTED;
+  FusedParams p;
+  p.sel.a = a;
+  p.sel.a.q_pooled = q_pooled; p.sel.a.k_pooled = k_pooled; p.sel.a.scores_in = nullptr; p.sel.a.refine = 0;
+  p.sel.status = ctx->d_status;
+  p.q = q.ptr; p.k = k.ptr;
+  p.q_sB = q.sB; p.q_sH = q.sH; p.q_sL = q.sL; p.k_sB = k.sB; p.k_sH = k.sH; p.k_sL = k.sL;
+  p.L_q = q.L; p.L_k = k.L; p.block = block;
+  p.vl = row_bytes / 16; p.groups = kThreads / p.vl;
+  p.first_k_block = first_k_block; p.k_cond_pooled = k_cond_pooled; p.n_cond = n_cond;
+  p.q_pooled = q_pooled; p.k_pooled = k_pooled;
+  return q.dtype == SPARSTAR_BF16 ? launch_fused_T<__nv_bfloat16>(ctx, p, s) : launch_fused_T<float>(ctx, p, s);
 }

@@ -57,6 +57,23 @@ class SparstarAttention:
                                  ratio=ratio, count=count, mass=mass, forced=forced, scores_out=scores)
         return num, idx, scores
 
+    def select_fused(self, q: torch.Tensor, k: torch.Tensor, block: int, mode: str, ratio: float = 0.0,
+                     count: int = 0, mass: float = 0.0, forced: Sequence[Tuple[int, int]] = (),
+                     scale: Optional[float] = None, cap: Optional[int] = None,
+                     k_cond_pooled: Optional[torch.Tensor] = None):
+        """pool(Q), pool(K), score + select in ONE launch.  Returns (kv_num_blocks, kv_indices)."""
+        scale = q.shape[3] ** -0.5 if scale is None else scale
+        B, H, L_q, D = q.shape
+        n_q, n_k = sp.sparstar_num_blocks(L_q, block), sp.sparstar_num_blocks(k.shape[2], block)
+        cap = n_k if cap is None else cap
+        qbar = torch.empty((B, H, n_q, D), dtype=torch.float32, device=q.device)
+        kbar = torch.empty((B, H, n_k, D), dtype=torch.float32, device=q.device)
+        num = torch.empty((B, H, n_q), dtype=torch.int32, device=q.device)
+        idx = torch.empty((B, H, n_q, cap), dtype=torch.int32, device=q.device)
+        sp.sparstar_select_fused(self.ctx, q, k, block, scale, _MODES[mode], qbar, kbar, num, idx, ratio=ratio,
+                                 count=count, mass=mass, forced=forced, k_cond_pooled=k_cond_pooled)
+        return num, idx
+
     def sparse_forward(self, q, k, v, block: int, kv_num_blocks, kv_indices, scale: Optional[float] = None,
                        want_lse: bool = False):
         scale = q.shape[3] ** -0.5 if scale is None else scale
@@ -195,18 +212,8 @@ class ClipPyramid:
         B, H, L_k, D = k.shape
         rho = self.density(q.shape[2])
         assert rho is not None, "this scale is not in the schedule (run it dense)"
-        n_q, n_k = sp.sparstar_num_blocks(q.shape[2], self.block), sp.sparstar_num_blocks(L_k, self.block)
-        qbar = self.eng.pool(q, self.block)
-        kbar = torch.empty((B, H, n_k, D), dtype=torch.float32, device=k.device)
-        fb = self.full_blocks if self.cond_pool is not None else 0
-        if fb > 0:
-            kbar[:, :, :fb].copy_(self.cond_pool)
-        sp.sparstar_pool_blocks_range(self.eng.ctx, k, self.block, fb, n_k - fb, kbar)
-        num = torch.empty((B, H, n_q), dtype=torch.int32, device=q.device)
-        idx = torch.empty((B, H, n_q, n_k), dtype=torch.int32, device=q.device)
-        sp.sparstar_score_select(self.eng.ctx, qbar, kbar, self.block, L_k, D ** -0.5, sp.SEL_TOPK_RATIO, num, idx,
-                                 ratio=rho, forced=self.forced)
-        return num, idx
+        cond = self.cond_pool if (self.cond_pool is not None and self.full_blocks > 0) else None
+        return self.eng.select_fused(q, k, self.block, "topk_ratio", ratio=rho, forced=self.forced, k_cond_pooled=cond)
 
     def forward(self, q, k, v):
         """One scale: sparse when the schedule lists its query length, dense otherwise."""

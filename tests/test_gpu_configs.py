@@ -249,3 +249,63 @@ def test_clip_pyramid_graph_replay(eng):
             want = pyr.forward(q, k, v)
             eng.check()
             assert torch.equal(o, want)
+
+
+def test_clip_pyramid_full_size_with_the_papers_schedule(eng):
+    """The four late scales of a later clip at full size (4,800 / 18,400 / 40,800 / 72,000 queries
+    against 72,512 conditioning keys + themselves, 32 heads) with the paper's density schedule
+    (0.625, 0.1875, 0.1875, 0.09375; clip >= 2: text kept, preceding-clip keys ranked jointly),
+    conditioning block means pooled once, one fused selection launch per scale: lists on sampled
+    heads and attention on sampled units against the oracle, then all four scales chained in one
+    CUDA graph and replayed."""
+    import paper_2608_10519_b200 as sp
+    from paper_2608_10519_b200.pipeline import ClipPyramid
+    scales = pyramid_sweep(0)
+    schedule = sp.sparstar_schedule_preset(sp.SCHEDULE_720P_PYRAMID)
+    assert [r for (_, r) in schedule] == [0.625, 0.1875, 0.1875, 0.09375]
+    w0 = scales[0]
+    text_len, ref_len = w0.segments[0].length, w0.segments[1].length
+    pyr = ClipPyramid(eng, 2, text_len, ref_len, w0.block, schedule, extra_forced=[(0, w0.n_sink)])
+    forced = orc.keep_ranges(2, (0, text_len), (text_len, text_len + ref_len)) + [(0, w0.n_sink)]
+    tau = w0.D ** -0.5
+    heads = (0, 31)
+    tensors = []
+    for w in scales:
+        x = generate(w, "cuda")
+        q, k, v = x["q"], x["k"], x["v"]
+        tensors.append((q, k, v))
+        if pyr.cond_pool is None:
+            pyr.set_conditioning(k[:, :, :text_len + ref_len])
+        else:                                              # the conditioning keys are the same at every scale of the clip
+            assert torch.equal(k[:, :, :text_len + ref_len], tensors[0][1][:, :, :text_len + ref_len])
+        rho = orc.density_lookup(schedule, w.L_q)
+        l0 = sp.sparstar_launch_count(eng.ctx)
+        num, idx = pyr.select(q, k)
+        assert sp.sparstar_launch_count(eng.ctx) - l0 == 1          # pooling + scores + selection: one launch
+        o, lse = eng.sparse_forward(q, k, v, w.block, num, idx, want_lse=True)
+        eng.check()
+        rep = compare.ListReport()
+        for h in heads:
+            lists, S, fm = orc.select_head(f64(q[0, h]), f64(k[0, h]), w.block, tau, forced, "topk_ratio", ratio=rho)
+            compare.compare_lists(num[0, h].cpu().numpy(), idx[0, h].cpu().numpy(), lists, S, fm, "topk_ratio",
+                                  k=orc.budget(int((~fm).sum()), rho), tag=f"{w.name} h{h}", report=rep)
+            Kh, Vh = f64(k[0, h]), f64(v[0, h])
+            got_lists = idx[0, h].cpu().numpy()
+            got_num = num[0, h].cpu().numpy()
+            for (_, i) in sample_units(w.n_q, 1, w.seed, 2, heads=(0,)):
+                r0, r1 = i * w.block, min((i + 1) * w.block, w.L_q)
+                want, want_lse = orc.attention_block(f64(q[0, h, r0:r1]), Kh, Vh, got_lists[i, :got_num[i]], w.block, tau)
+                compare.check_output(f64(o[0, h, r0:r1]), want, "bf16", f"{w.name} h{h} i{i}")
+                assert np.abs(f64(lse[0, h, r0:r1]) - want_lse).max() <= 1e-3
+        print(f"{w.name}: rho {rho}: rows {rep.rows} exact {rep.exact} excused {rep.excused}")
+        assert rep.ok and rep.exact == rep.rows, rep.bad[:3]      # exact lists: the outputs above were formed with the oracle's lists
+    # the whole clip as one graph
+    eager = [pyr.forward(q, k, v) for (q, k, v) in tensors]
+    graph, outs = pyr.capture(tensors)
+    for o_ in outs:
+        o_.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    eng.check()
+    for a, b in zip(eager, outs):
+        assert torch.equal(a, b)

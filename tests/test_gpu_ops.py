@@ -709,3 +709,30 @@ def test_context_checks_the_current_device(eng):
     out = eng.pool(x, 128)
     eng.check()
     assert out.shape == (1, 1, 2, 128)
+
+
+@pytest.mark.parametrize("mode,kw", [("topk_ratio", {"ratio": 0.25}), ("mass", {"mass": 0.9}), ("topk_count", {"count": 3})])
+def test_select_fused_gives_the_lists_of_the_separate_calls(eng, mode, kw):
+    """Pooling + scores + selection in one cooperative launch: the same bits as pool, pool,
+    score_select, with and without cached block means of the leading (conditioning) key blocks."""
+    for (dtype, D, block, H, L_q, L_k) in [(torch.bfloat16, 128, 128, 3, 128 * 11 + 70, 128 * 37 + 5),
+                                           (torch.float32, 64, 64, 2, 64 * 5 + 1, 64 * 9)]:
+        q, k = _rand((1, H, L_q, D), dtype, 900), _rand((1, H, L_k, D), dtype, 901)
+        forced = [(0, block + 7)]
+        want_num, want_idx, _ = eng.select(q, k, block, mode, forced=forced, **kw)
+        num, idx = eng.select_fused(q, k, block, mode, forced=forced, **kw)
+        eng.check()
+        assert torch.equal(num, want_num)
+        for h in range(H):
+            for i in range(num.shape[2]):
+                c = int(num[0, h, i])
+                assert torch.equal(idx[0, h, i, :c], want_idx[0, h, i, :c])
+        # the first 5 key blocks from a cache
+        cond = eng.pool(k[:, :, :5 * block], block)
+        num2, idx2 = eng.select_fused(q, k, block, mode, forced=forced, k_cond_pooled=cond, **kw)
+        eng.check()
+        assert torch.equal(num2, want_num)
+        for h in range(H):
+            for i in range(num.shape[2]):
+                c = int(num[0, h, i])
+                assert torch.equal(idx2[0, h, i, :c], want_idx[0, h, i, :c])
