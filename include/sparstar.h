@@ -255,7 +255,8 @@ int sparstar_attn_fwd(sparstar_ctx* ctx, const sparstar_tensor* q, const sparsta
  * sparstar_block_mass: exact post-softmax mass per (query block, key block),
  *   M_ij = mean over queries t of block i of sum over keys u of block j of softmax_u(scale q_t.k_u),
  *   from Q, K and the log-sum-exp of the dense attention (`lse_dense` [B,H,L_q], as written by
- *   sparstar_attn_fwd).  mass_out [B,H,n_q,n_k] fp32, rows sum to 1.  bf16, D = 128, block = 128.
+ *   sparstar_attn_fwd).  mass_out [B,H,n_q,n_k] fp32 (n = ceil(L / block)), rows sum to 1.  bf16, D in
+ *   {64, 128}, block in {32, 64, 128, 256, 512}.
  * sparstar_select_from_scores: the selection stage of sparstar_score_select applied to a given
  *   score array [B,H,n_q,n_k] fp32 (e.g. the exact masses: the block-wise oracle selector of
  *   the paper's analysis) with the same params, tie rule, forced blocks and outputs.

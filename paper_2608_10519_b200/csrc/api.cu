@@ -417,9 +417,10 @@ int sparstar_block_mass(sparstar_ctx* ctx, const sparstar_tensor* q, const spars
   int st;
   if ((st = check_tensor(q)) || (st = check_tensor(k))) return st;
   if (k->B != q->B || k->H != q->H || k->D != q->D || k->dtype != q->dtype) return SPARSTAR_ERR_INVALID_ARG;
-  if (q->dtype != SPARSTAR_BF16 || q->D != 128 || block != 128 || q->H > 65535 || q->B > 65535)
+  const bool block_ok = block == 32 || block == 64 || block == 128 || block == 256 || block == 512;
+  if (q->dtype != SPARSTAR_BF16 || (q->D != 128 && q->D != 64) || !block_ok || q->H > 65535 || q->B > 65535)
     return SPARSTAR_ERR_UNSUPPORTED;
-  return launch_block_mass_tc(ctx, *q, *k, scale, lse_dense, mass_out, static_cast<cudaStream_t>(stream));
+  return launch_block_mass_tc(ctx, *q, *k, block, scale, lse_dense, mass_out, static_cast<cudaStream_t>(stream));
 }
 
 int sparstar_retained_mass(sparstar_ctx* ctx, const float* mass, const int32_t* kv_num_blocks,

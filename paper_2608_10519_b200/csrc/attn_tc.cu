@@ -325,9 +325,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bool ok = true;
     const int n_mine = (n - x + 1) / 2;             // list positions x, x+2, ...
     float mass_lse2 = 0.f, mass_w = 0.f;
+    // mass mode: the selection block this row belongs to (blocks of 128 * m tokens, or p.mass_g blocks
+    // of 128 / mass_g tokens per tile; rows of one warp share a block) and its count of valid queries
+    int mass_qb = 0;
     if (kMass) {
       const int q_row = qi * kBlock + row;
-      const int q_valid = min(kBlock, p.L_q - qi * kBlock);
+      const int blk_len = p.mass_g > 1 ? kBlock / p.mass_g : kBlock * p.m;
+      mass_qb = q_row / blk_len;
+      const int q_valid = min(blk_len, p.L_q - mass_qb * blk_len);
       if (q_row < p.L_q) {
         mass_lse2 = p.lse_in[((size_t)b * p.H + h) * p.L_q + q_row] * 1.4426950408889634f;
         mass_w = 1.0f / (float)q_valid;
@@ -401,18 +406,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       load_s();
       TRACE(1 + x, 31, t);
       if (kMass) {
-        // p = exp(scale*s - lse_row): the dense softmax probability; sum over the tile's keys
+        // p = exp(scale*s - lse_row): the dense softmax probability, summed over the keys of each 32-column
+        // segment of the tile, then over the segments of one key block
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int i = 0; i < 128; ++i) acc[i & 3] += ex2(fmaf(__uint_as_float(sr[i]), c, -mass_lse2));
-        float rs = ((acc[0] + acc[1]) + (acc[2] + acc[3])) * mass_w;     // rows past L_q weigh 0
+        for (int sgm = 0; sgm < 4; ++sgm)
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) rs += __shfl_xor_sync(0xffffffffu, rs, o);
-        // one atomic per warp into the zero-initialised output: no barrier inside the loop, so a
-        // warp that abandons a wait can never leave the others of its warpgroup stranded
-        if (lane == 0) {
-          const int j = dense ? t : min(max(list[t], 0), p.n_k - 1);
-          atomicAdd(&p.mass_out[row_id * (size_t)p.n_k + j], rs);
+          for (int i = 0; i < 32; ++i) acc[sgm] += ex2(fmaf(__uint_as_float(sr[32 * sgm + i]), c, -mass_lse2));
+        const int g = p.mass_g;                                          // key blocks per tile
+        float rs[4];
+        if (g == 1) { rs[0] = (acc[0] + acc[1]) + (acc[2] + acc[3]); rs[1] = rs[2] = rs[3] = 0.f; }
+        else if (g == 2) { rs[0] = acc[0] + acc[1]; rs[1] = acc[2] + acc[3]; rs[2] = rs[3] = 0.f; }
+        else { rs[0] = acc[0]; rs[1] = acc[1]; rs[2] = acc[2]; rs[3] = acc[3]; }
+        const int tile = dense ? t : min(max(list[t], 0), p.n_k - 1);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (e < g) {
+            float v_ = rs[e] * mass_w;                                   // rows past L_q weigh 0
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v_ += __shfl_xor_sync(0xffffffffu, v_, o);
+            // one atomic per warp and key block into the zero-initialised output: no barrier inside the
+            // loop, so a warp that abandons a wait can never leave the others of its warpgroup stranded
+            const int kb = g > 1 ? tile * g + e : tile / p.m;
+            if (lane == 0 && kb < p.n_kb && mass_qb < p.n_qb)
+              atomicAdd(&p.mass_out[(((size_t)b * p.H + h) * p.n_qb + mass_qb) * (size_t)p.n_kb + kb], v_);
+          }
         }
         mbar_arrive(bar(BAR_PFULL + x));                                 // S may be overwritten
         continue;
@@ -693,7 +711,7 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   p.scale = a.scale;
   p.kv_num_blocks = a.kv_num_blocks; p.kv_indices = a.kv_indices; p.cap = a.cap;
   p.lse = a.lse;
-  p.lse_in = nullptr; p.mass_out = nullptr;
+  p.lse_in = nullptr; p.mass_out = nullptr; p.mass_g = 1;
   p.order = nullptr;
   const bool want_order = !dense && p.n_q > 1 && (size_t)p.n_q * sizeof(int) <= 200 * 1024 &&
                           ctx->debug_work_order != 0;
@@ -755,7 +773,7 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
 }
 
 // ---- block attention mass (analysis) --------------------------------------------------------
-int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const sparstar_tensor& k, float scale,
+int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const sparstar_tensor& k, int block, float scale,
                          const float* lse_dense, float* mass_out, cudaStream_t s) {
   CUtensorMap mq, mk;
   int st;
@@ -763,9 +781,13 @@ int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const spar
   TcParams p;
   p.o = nullptr; p.osB = p.osH = p.osL = 0;
   p.H = q.H; p.L_q = q.L; p.L_k = k.L;
-  p.n_q = (q.L + kBlock - 1) / kBlock;
+  p.n_q = (q.L + kBlock - 1) / kBlock;                    // 128-token tiles: the kernel walks every (query tile, key tile)
   p.n_k = (k.L + kBlock - 1) / kBlock;
-  p.m = 1; p.n_qb = p.n_q; p.n_kb = p.n_k; p.gather = 1;
+  p.n_qb = (q.L + block - 1) / block;                     // the output is per selection block
+  p.n_kb = (k.L + block - 1) / block;
+  p.m = block >= kBlock ? block / kBlock : 1;
+  p.mass_g = block < kBlock ? kBlock / block : 1;
+  p.gather = 1;
   p.scale = scale;
   p.kv_num_blocks = nullptr; p.kv_indices = nullptr; p.cap = 0;
   p.lse = nullptr;
@@ -775,8 +797,8 @@ int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const spar
   p.trace = nullptr; p.trace_cap = 0; p.trace_skip = 0;
   p.debug_drop_stage = -1;
   dim3 grid(p.n_q, q.H, q.B);
-  SPARSTAR_CUDA_TRY(cudaMemsetAsync(mass_out, 0, sizeof(float) * (size_t)q.B * q.H * p.n_q * p.n_k, s));
-  st = launch_variant<1>(ctx, mq, mk, mk, p, grid, s);
+  SPARSTAR_CUDA_TRY(cudaMemsetAsync(mass_out, 0, sizeof(float) * (size_t)q.B * q.H * p.n_qb * p.n_kb, s));
+  st = q.D == 64 ? launch_variant<1, 64>(ctx, mq, mk, mk, p, grid, s) : launch_variant<1, 128>(ctx, mq, mk, mk, p, grid, s);
   if (st != SPARSTAR_OK) return st;
   ctx->launches++;
   SPARSTAR_CUDA_TRY(cudaGetLastError());
@@ -862,7 +884,7 @@ extern "C" int sparstar_sparse_attn_fwd_static(const sparstar_tensor* q, const s
   p.scale = scale;
   p.kv_num_blocks = kv_num_blocks; p.kv_indices = kv_indices; p.cap = cap;
   p.lse = lse;
-  p.lse_in = nullptr; p.mass_out = nullptr;
+  p.lse_in = nullptr; p.mass_out = nullptr; p.mass_g = 1;
   p.order = scratch->order;
   p.status = status;
   p.trace = nullptr; p.trace_cap = 0; p.trace_skip = 0;

@@ -65,7 +65,8 @@ struct TcParams {
   const int* kv_indices;
   int cap;
   const float* lse_in;   // mass mode: [B,H,L_q] log-sum-exp of the dense attention (natural log)
-  float* mass_out;       // mass mode: [B,H,n_q,n_k]
+  float* mass_out;       // mass mode: [B,H,n_qb,n_kb] (per selection block)
+  int mass_g;            // mass mode: selection blocks per 128-token tile (1, or 2 / 4 for blocks of 64 / 32 tokens)
   const int* order;      // optional [B*H][n_q]: query blocks of each head, longest list first
   float* lse;
   sparstar_devstatus* status;

@@ -103,7 +103,7 @@ struct AttnArgs {
 int launch_attn_simt(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s);
 bool attn_tc_supported(const AttnArgs& a);
-int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const sparstar_tensor& k, float scale,
+int launch_block_mass_tc(sparstar_ctx* ctx, const sparstar_tensor& q, const sparstar_tensor& k, int block, float scale,
                          const float* lse_dense, float* mass_out, cudaStream_t s);
 int launch_retained_mass(sparstar_ctx* ctx, const float* mass, const int* kv_num_blocks, const int* kv_indices,
                          int rows, int n_k, int cap, float* out, cudaStream_t s);
