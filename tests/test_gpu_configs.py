@@ -86,7 +86,7 @@ def _full_size_case(eng, w, sel_heads, n_hashed, attn_heads=None, dense_units=0)
         for i in range(0, w.n_q, max(1, w.n_q // 50)):
             row = idx_h[h, i, :num_h[h, i]]
             assert np.all(np.diff(row) > 0) and set(f_ids) <= set(row)
-        for i, l in enumerate(lists):                      # outputs are judged with the oracle's lists
+        for i, l in enumerate(lists):                      # the attention below runs with the oracle's lists
             num_o[h, i] = len(l)
             idx_o[h, i, :len(l)] = l
     print(f"{w.name}: lists on {len(sel_heads)} heads: rows {rep.rows} exact {rep.exact} excused {rep.excused}")

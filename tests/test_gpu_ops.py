@@ -173,6 +173,14 @@ def test_attention_tcgen05(eng, L_q, L_k, H, density):
     _attn_case(eng, torch.bfloat16, 128, 128, L_q, L_k, H, density, 13, 2)
 
 
+@pytest.mark.parametrize("D,L_q,L_k,H,density", [(128, 128 * 2 + 96, 128 * 6 + 32, 2, 0.4), (128, 128 * 5, 128 * 33, 2, 0.15),
+                                                 (64, 128 * 3, 128 * 20, 2, 0.2), (128, 128, 128, 1, 1.0)])
+def test_attention_two_stream_kernel_cross_check(eng, D, L_q, L_k, H, density):
+    """The older two-stream kernel (two score tiles, two accumulators merged at the end), selectable
+    as ATTN_TCGEN05_2STREAM: the same oracle, an independent pipeline."""
+    _attn_case(eng, torch.bfloat16, D, 128, L_q, L_k, H, density, 17, 3)
+
+
 def test_attention_tcgen05_strided_inputs_and_rerun(eng):
     """Non-contiguous views (packed QKV-style buffer) and bit-reproducibility of two runs."""
     import paper_2608_10519_b200 as sp
