@@ -84,7 +84,6 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + kOff3Misc);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + kOff3Misc + 4);
-  volatile float* lsum = reinterpret_cast<volatile float*>(tail + kOff3Lsum);
   volatile float* mref = reinterpret_cast<volatile float*>(tail + kOff3Mref);
   volatile uint32_t* trace_smem = reinterpret_cast<volatile uint32_t*>(tail + kOff3Trace);
 
@@ -382,36 +381,55 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), (uint32_t)((n - 1) / 3 + 1) & 1u, abort_flag, 320 + w));
       tc_fence_after();
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");            // every row's last reference is published
-    const float ref = mref[row];
-    lsum[w * 128 + row] = my_ref > -INFINITY ? l * ex2((my_ref - ref) * c) : 0.f;
+    // The K/V rings are dead now (every service of this CTA is complete) and serve as scratch: the row's two
+    // partial results meet there, and the output is staged there so that it leaves in whole 128-byte row
+    // pieces instead of 32 scattered 16-byte pieces per store instruction.
+    unsigned char* vring = smem_raw + kOffV;
+    volatile float* stats = reinterpret_cast<volatile float*>(vring + 32768);   // (reference, partial denominator)
+    stats[2 * (w * 128 + row)] = my_ref;
+    stats[2 * (w * 128 + row) + 1] = l;
     asm volatile("bar.sync 1, 256;" ::: "memory");
     const int q_row = q_row0 + row;
     constexpr int kCols = HD / 2;                   // this warpgroup's half of D
     constexpr int kChunks = kCols / 32;
     if (*abort_flag == 0 && n > 0) {
-      const float lt = lsum[row] + lsum[128 + row];
+      // references only rise, so the row's final reference is the larger of the two cached ones
+      const float oref = stats[2 * ((w ^ 1) * 128 + row)], ol = stats[2 * ((w ^ 1) * 128 + row) + 1];
+      const float ref = fmaxf(my_ref, oref);
+      const float lt = (my_ref > -INFINITY ? l * ex2((my_ref - ref) * c) : 0.f) +
+                       (oref > -INFINITY ? ol * ex2((oref - ref) * c) : 0.f);
       const float inv = lt > 0.f ? 1.0f / lt : 0.f;
       const uint32_t col0 = (uint32_t)w * (uint32_t)kCols;
       uint32_t oa[kChunks][32];
 #pragma unroll
       for (int cc = 0; cc < kChunks; ++cc) tmem_ld32(tO + lane_off + col0 + 32u * cc, oa[cc]);
       tmem_wait_ld();
-      if (q_row < p.L_q) {
-        __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o) + b * p.osB + h * p.osH +
-                            (long long)q_row * p.osL + col0;
-        uint32_t out[kChunks * 16];
+      // this warp's 32 rows x kCols columns, staged with the 16-byte pieces of a row rotated by the row number
+      // (no bank conflicts either way), then stored row-contiguously
+      constexpr int kRowBytes = kCols * 2;
+      constexpr int kPieces = kRowBytes / 16;       // 8 (D = 128) or 4 (D = 64)
+      unsigned char* stage = vring + warp * (32 * kRowBytes);
 #pragma unroll
-        for (int cc = 0; cc < kChunks; ++cc)
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            out[cc * 16 + i] = pack_bf16(__uint_as_float(oa[cc][2 * i]) * inv, __uint_as_float(oa[cc][2 * i + 1]) * inv);
-        uint4* dst = reinterpret_cast<uint4*>(og);
-#pragma unroll
-        for (int i = 0; i < kChunks * 4; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
-        if (p.lse != nullptr && w == 0)
-          p.lse[((size_t)b * p.H + h) * p.L_q + q_row] = lt > 0.f ? ref * p.scale + logf(lt) : -INFINITY;
+      for (int pc = 0; pc < kPieces; ++pc) {
+        const uint32_t* src = &oa[pc / 4][8 * (pc % 4)];
+        uint4 val;
+        val.x = pack_bf16(__uint_as_float(src[0]) * inv, __uint_as_float(src[1]) * inv);
+        val.y = pack_bf16(__uint_as_float(src[2]) * inv, __uint_as_float(src[3]) * inv);
+        val.z = pack_bf16(__uint_as_float(src[4]) * inv, __uint_as_float(src[5]) * inv);
+        val.w = pack_bf16(__uint_as_float(src[6]) * inv, __uint_as_float(src[7]) * inv);
+        *reinterpret_cast<uint4*>(stage + lane * kRowBytes + ((pc ^ (lane & (kPieces - 1))) * 16)) = val;
       }
+      __syncwarp();
+      __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(p.o) + b * p.osB + h * p.osH + col0;
+      const int warp_row0 = q_row0 + (warp & 3) * 32;
+#pragma unroll
+      for (int i = 0; i < kPieces; ++i) {
+        const int r = i * (32 / kPieces) + lane / kPieces, pc = lane % kPieces;
+        const uint4 val = *reinterpret_cast<const uint4*>(stage + r * kRowBytes + ((pc ^ (r & (kPieces - 1))) * 16));
+        if (warp_row0 + r < p.L_q) *reinterpret_cast<uint4*>(ob + (long long)(warp_row0 + r) * p.osL + pc * 8) = val;
+      }
+      if (q_row < p.L_q && p.lse != nullptr && w == 0)
+        p.lse[((size_t)b * p.H + h) * p.L_q + q_row] = lt > 0.f ? ref * p.scale + logf(lt) : -INFINITY;
     } else if (n == 0 && live) {
       if (q_row < p.L_q) {
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o) + b * p.osB + h * p.osH +
