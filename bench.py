@@ -479,6 +479,9 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
     ap.add_argument("--block", type=int, default=0, help="override the workload's selection block size (profiling captures)")
     ap.add_argument("--impl", default="sparstar", choices=["sparstar", "reference"])
+    ap.add_argument("--attn-impl", type=int, default=0,
+                    help="attention implementation of the library (sparstar_attn_impl; 0 = default, 4 = CTA pairs where "
+                         "two query tiles share a list: the dense comparison and blocks of 256 / 512 tokens)")
     ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
                     help="N > 1: weak = one workload per GPU (default), strong = the heads of one workload split across GPUs")
     ap.add_argument("--no-library-dense", action="store_true", help="skip the torch SDPA / FlashAttention-2 dense timings")
@@ -531,6 +534,8 @@ def main():
         x = generate(w, dev)
     q, k, v = x["q"], x["k"], x["v"]
     eng = SparstarAttention(local)
+    if args.attn_impl:
+        sp.sparstar_set_attn_impl(eng.ctx, args.attn_impl)
     ctx = eng.ctx
     B, H, D, blk = w.B, w.H, w.D, w.block
     scale = D ** -0.5

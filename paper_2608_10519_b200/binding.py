@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libsparstar.so")
 
 F32, BF16 = 0, 1
 SEL_TOPK_RATIO, SEL_TOPK_COUNT, SEL_MASS = 0, 1, 2
-ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_2STREAM = 0, 1, 2, 3
+ATTN_AUTO, ATTN_SIMT, ATTN_TCGEN05, ATTN_TCGEN05_2STREAM, ATTN_TCGEN05_PAIR = 0, 1, 2, 3, 4
 SCORE_FP64, SCORE_TCGEN05 = 0, 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_BAD_INDEX, ERR_TIMEOUT, ERR_CUDA, ERR_TOO_LARGE, ERR_CAPTURE = range(9)
 

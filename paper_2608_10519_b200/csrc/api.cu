@@ -80,7 +80,7 @@ int check_attn(const sparstar_tensor* q, const sparstar_tensor* k, const sparsta
 
 int dispatch_attn(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   const int impl = ctx->attn_impl;
-  if (impl == SPARSTAR_ATTN_TCGEN05 || impl == SPARSTAR_ATTN_TCGEN05_2STREAM) {
+  if (impl == SPARSTAR_ATTN_TCGEN05 || impl == SPARSTAR_ATTN_TCGEN05_2STREAM || impl == SPARSTAR_ATTN_TCGEN05_PAIR) {
     if (!attn_tc_supported(a)) return SPARSTAR_ERR_UNSUPPORTED;
     return launch_attn_tc(ctx, a, s);
   }
@@ -183,7 +183,7 @@ int sparstar_check(sparstar_ctx* ctx, void* stream, int32_t* site) {
 }
 
 int sparstar_set_attn_impl(sparstar_ctx* ctx, int32_t impl) {
-  if (ctx == nullptr || impl < SPARSTAR_ATTN_AUTO || impl > SPARSTAR_ATTN_TCGEN05_2STREAM)
+  if (ctx == nullptr || impl < SPARSTAR_ATTN_AUTO || impl > SPARSTAR_ATTN_TCGEN05_PAIR)
     return SPARSTAR_ERR_INVALID_ARG;
   ctx->attn_impl = impl;
   return SPARSTAR_OK;

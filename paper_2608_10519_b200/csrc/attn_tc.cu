@@ -698,7 +698,11 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   const int gather = !dense && a.block < kBlock ? kBlock / a.block : 1;
   const int block = dense ? kBlock : a.block;
   const int kv_rows = kBlock / gather;
-  if ((st = make_map(&mq, a.q)) || (st = make_map(&mk, a.k, kv_rows)) || (st = make_map(&mv, a.v, kv_rows))) return st;
+  // two adjacent query tiles on a pair of CTAs: they must walk the same list
+  const bool pair = ctx->attn_impl == SPARSTAR_ATTN_TCGEN05_PAIR && gather == 1 && a.q.D == 128 &&
+                    (dense || (block / kBlock) % 2 == 0);
+  if ((st = make_map(&mq, a.q)) || (st = make_map(&mk, a.k, pair ? 64 : kv_rows)) || (st = make_map(&mv, a.v, kv_rows)))
+    return st;
   TcParams p;
   p.o = a.o.ptr; p.osB = a.o.sB; p.osH = a.o.sH; p.osL = a.o.sL;
   p.H = a.q.H; p.L_q = a.q.L; p.L_k = a.k.L;
@@ -750,8 +754,10 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
       SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
       order_attr[ctx->device & 63] = true;
     }
-    attn_order_kernel<<<a.q.B * a.q.H, 256, (size_t)p.n_q * sizeof(int), s>>>(p.kv_num_blocks, p.n_q, p.m, p.n_qb,
-                                                                               p.cap, order);
+    // work items: query tiles, or (CTA pairs) pairs of adjacent tiles of one selection block
+    const int n_items = pair ? (p.n_q + 1) / 2 : p.n_q, per_block = pair ? p.m / 2 : p.m;
+    attn_order_kernel<<<a.q.B * a.q.H, 256, (size_t)n_items * sizeof(int), s>>>(p.kv_num_blocks, n_items, per_block,
+                                                                                 p.n_qb, p.cap, order);
     ctx->launches++;
     p.order = order;
   }
@@ -765,7 +771,7 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   else if (ctx->attn_impl == SPARSTAR_ATTN_TCGEN05_2STREAM)
     st2 = a.q.D == 64 ? launch_variant<0, 64>(ctx, mq, mk, mv, p, grid, s) : launch_variant<0, 128>(ctx, mq, mk, mv, p, grid, s);
   else
-    st2 = launch_attn_tc3(ctx, mq, mk, mv, p, a.q.D, grid, s);
+    st2 = launch_attn_tc3(ctx, mq, mk, mv, p, a.q.D, grid, s, pair);
   if (st2 != SPARSTAR_OK) return st2;
   ctx->launches++;
   SPARSTAR_CUDA_TRY(cudaGetLastError());

@@ -49,30 +49,44 @@ enum {
   B3_STAGE = 1,             // 3
   B3_SFULL = B3_STAGE + 3,  // 3
   B3_PFULL = B3_SFULL + 3,  // 3
-  B3_COUNT = B3_PFULL + 3
+  // CTA pairs only, used in the first CTA: what the second CTA contributes is counted on barriers of its own
+  B3_PEERP = B3_PFULL + 3,       // 3: the second CTA's warps have written their P
+  B3_PEERQ = B3_PEERP + 3,       // the second CTA's Q and its halves of the first K tiles
+  B3_PEERSTAGE = B3_PEERQ + 1,   // 3: the second CTA's halves of {V_u, K_{u+3}}
+  B3_COUNT = B3_PEERSTAGE + 3
 };
 constexpr float kRaiseLog2 = 52.5f;   // a tile whose row maximum exceeds the reference by more than 2^52.5 raises it
                                       // (128 exponentials of at most 2^53 sum to at most kSumLimit = 2^60)
 
-constexpr uint32_t smem3_tiles(int hd) { return (1u + 2u * kStages) * (128u * (uint32_t)hd * 2u); }
-constexpr uint32_t kOff3Misc = 8u * 16u;                         // after the barrier area (16 slots)
+// Q, then kStages slots of K and of V; a CTA of a pair holds half of every K and V tile
+constexpr uint32_t smem3_tiles(int hd, bool pair = false) {
+  return (1u + (pair ? 1u : 2u) * kStages) * (128u * (uint32_t)hd * 2u);
+}
+constexpr uint32_t kOff3Misc = 8u * 24u;                         // after the barrier area (24 slots)
 constexpr uint32_t kOff3Lsum = kOff3Misc + 16u;                  // 2 x 128 floats: partial denominators at the final reference
 constexpr uint32_t kOff3Mref = kOff3Lsum + 2u * 128u * 4u;       // 128 floats: the rows' published references
 constexpr uint32_t kOff3Trace = kOff3Mref + 128u * 4u;
 constexpr uint32_t kTail3Bytes = kOff3Trace + 4u * kTraceSlots * 4u;
-constexpr uint32_t smem3_bytes(int hd) { return smem3_tiles(hd) + kTail3Bytes; }
-static_assert(B3_COUNT <= 16, "barrier area");
+// A CTA of a pair has an epilogue scratch of its own behind the tail (34 KB used); a single CTA reuses its V ring
+constexpr uint32_t kTail3Padded = (kTail3Bytes + 1023u) & ~1023u;
+constexpr uint32_t kPairScratch = 36u * 1024u;
+constexpr uint32_t smem3_bytes(int hd, bool pair = false) {
+  return smem3_tiles(hd, pair) + (pair ? kTail3Padded + kPairScratch : kTail3Bytes);
+}
+static_assert(B3_COUNT <= 24, "barrier area");
 static_assert(smem3_bytes(128) <= 232448u, "shared memory per CTA");
 
-template <int HD>
+template <int HD, bool kPair, bool kTrace>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const TcParams p) {
   static_assert(HD == 64 || HD == 128, "head dimension");
+  static_assert(!kPair || HD == 128, "CTA pairs: head dimension 128");
   constexpr uint32_t kTileBytes = 128u * HD * 2u;
+  constexpr uint32_t kKVBytes = kPair ? kTileBytes / 2u : kTileBytes;   // this CTA's share of a K or V tile
   constexpr uint32_t kOffK = kOffQ + kTileBytes;
-  constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
-  constexpr uint32_t kOffTail = kOffV + kStages * kTileBytes;
+  constexpr uint32_t kOffV = kOffK + kStages * kKVBytes;
+  constexpr uint32_t kOffTail = kOffV + kStages * kKVBytes;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   unsigned char* tail = smem_raw + kOffTail;
@@ -88,14 +102,21 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   volatile uint32_t* trace_smem = reinterpret_cast<volatile uint32_t*>(tail + kOff3Trace);
 
   const int h = blockIdx.y, b = blockIdx.z;
-  int qi = p.order != nullptr ? p.order[((size_t)b * p.H + h) * p.n_q + blockIdx.x] : (int)blockIdx.x;
-  if (qi < 0 || qi >= p.n_q) {      // a work order that is not this launch's (stale scratch): flag it, stay in bounds
+  // work item: a query tile, or (CTA pairs) two adjacent query tiles that walk the same list
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;
+  const int item = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_items = kPair ? (p.n_q + 1) / 2 : p.n_q;
+  int wi = p.order != nullptr ? p.order[((size_t)b * p.H + h) * n_items + item] : item;
+  if (wi < 0 || wi >= n_items) {    // a work order that is not this launch's (stale scratch): flag it, stay in bounds
     if (threadIdx.x == 0) record_status(p.status, SPARSTAR_ERR_BAD_INDEX, -1);
-    qi = (int)blockIdx.x;
+    wi = item;
   }
+  // the second CTA of the last pair of an odd number of tiles gets a tile past the end: zero-filled Q, no output
+  const int qi = kPair ? 2 * wi + (int)rank : wi;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const size_t row_id = ((size_t)b * p.H + h) * p.n_qb + qi / p.m;      // the query block's list
-  const bool tracing = p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0 &&
+  const size_t row_id = ((size_t)b * p.H + h) * p.n_qb + (kPair ? 2 * wi : qi) / p.m;      // the query block's list
+  // clock stamps cost registers in the softmax loop: they exist only in the instances launched with a trace buffer
+  const bool tracing = kTrace && p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && lane == 0 &&
                        (warp == 0 || warp == 4 || warp >= 8);
   int trace_n = 0;
   const bool dense = p.kv_num_blocks == nullptr;
@@ -112,19 +133,28 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       mbar_init(bar(B3_STAGE + i), 1);
       mbar_init(bar(B3_SFULL + i), 1);
       mbar_init(bar(B3_PFULL + i), 4);
+      if (kPair) {
+        mbar_init(bar(B3_PEERP + i), 4);
+        mbar_init(bar(B3_PEERSTAGE + i), 1);
+      }
     }
+    if (kPair) mbar_init(bar(B3_PEERQ), 1);
     // an expired wait already on record (this launch or an earlier one): do no work, so that a
     // failing launch ends after one timeout instead of one per wave of CTAs
     *abort_flag = *reinterpret_cast<volatile int*>(&p.status->status) == SPARSTAR_ERR_TIMEOUT ? 1 : 0;
-    if (p.trace != nullptr)
+    if (kTrace && p.trace != nullptr)
       for (int i = 0; i < 4 * kTraceSlots; ++i) trace_smem[i] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (threadIdx.x < 128) mref[threadIdx.x] = -INFINITY;
-  if (warp == 9) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  if (warp == 9) {
+    if (kPair) tmem_alloc_pair(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+    else tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();     // both CTAs' barriers exist before either signals the other's
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tS[3] = {tmem + 0u, tmem + 128u, tmem + 256u};
@@ -152,17 +182,59 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const int j = checked(list[p.m == 1 ? t : t / p.m], sub == 0);
         return min(j * p.m + sub, p.n_k - 1) * kBlock;
       };
-      auto load_tile = [&](const CUtensorMap* map, uint32_t dst, uint32_t barrier, int row) {
-        tma_load_4d(dst, map, barrier, 0, row, h, b);
-        if (HD == 128) tma_load_4d(dst + kHalfBytes, map, barrier, 64, row, h, b);
+      // A CTA of a pair copies its own query tile, keys [64 rank, 64 rank + 64) of every K tile and columns
+      // [64 rank, 64 rank + 64) of every V tile.  The first CTA's bytes are counted on its barriers Q / STAGE, the
+      // second CTA's on the first CTA's barriers PEERQ / PEERSTAGE; the first CTA's producer arms both (the two
+      // CTAs copy the same amounts).
+      auto peer_of = [&](int i) { return i == B3_Q ? (int)B3_PEERQ : (int)B3_PEERSTAGE + (i - (int)B3_STAGE); };
+      auto barrier_of = [&](int i) { return kPair && rank == 1u ? cluster_map(bar(peer_of(i)), 0u) : bar(i); };
+      auto arm = [&](int i, uint32_t bytes) {          // `bytes`: what ONE CTA copies
+        if (rank == 0u) {
+          mbar_expect_tx(bar(i), bytes);
+          if (kPair) mbar_expect_tx(bar(peer_of(i)), bytes);
+        }
+      };
+      auto load_q = [&](int bi) {
+        const uint32_t dst = base + kOffQ, bb = barrier_of(bi);
+        if (kPair && rank == 1u) {
+          tma_load_4d_pair(dst, &map_q, bb, 0, q_row0, h, b);
+          tma_load_4d_pair(dst + kHalfBytes, &map_q, bb, 64, q_row0, h, b);
+        } else {
+          tma_load_4d(dst, &map_q, bb, 0, q_row0, h, b);
+          if (HD == 128) tma_load_4d(dst + kHalfBytes, &map_q, bb, 64, q_row0, h, b);
+        }
+      };
+      auto load_k = [&](int slot, int bi, int row) {
+        const uint32_t dst = base + kOffK + (uint32_t)slot * kKVBytes, bb = barrier_of(bi);
+        if (kPair && rank == 1u) {                         // 64 keys x D as two boxes of 64 x 64 (map with 64-row boxes)
+          tma_load_4d_pair(dst, &map_k, bb, 0, row + 64, h, b);
+          tma_load_4d_pair(dst + kKVBytes / 2u, &map_k, bb, 64, row + 64, h, b);
+        } else if (kPair) {
+          tma_load_4d(dst, &map_k, bb, 0, row, h, b);
+          tma_load_4d(dst + kKVBytes / 2u, &map_k, bb, 64, row, h, b);
+        } else {
+          tma_load_4d(dst, &map_k, bb, 0, row, h, b);
+          if (HD == 128) tma_load_4d(dst + kHalfBytes, &map_k, bb, 64, row, h, b);
+        }
+      };
+      auto load_v = [&](int slot, int bi, int row) {
+        const uint32_t dst = base + kOffV + (uint32_t)slot * kKVBytes, bb = barrier_of(bi);
+        if (kPair && rank == 1u) {                         // 128 keys x 64 columns: one box
+          tma_load_4d_pair(dst, &map_v, bb, 64, row, h, b);
+        } else if (kPair) {
+          tma_load_4d(dst, &map_v, bb, 0, row, h, b);
+        } else {
+          tma_load_4d(dst, &map_v, bb, 0, row, h, b);
+          if (HD == 128) tma_load_4d(dst + kHalfBytes, &map_v, bb, 64, row, h, b);
+        }
       };
       // Q with the first three score tiles' keys
       int jt[3] = {0, 0, 0};
       const int n_pro = min(n, 3);
       for (int t = 0; t < n_pro; ++t) jt[t] = block_at(t);
-      mbar_expect_tx(bar(B3_Q), kTileBytes * (uint32_t)(1 + n_pro));
-      load_tile(&map_q, base + kOffQ, bar(B3_Q), q_row0);
-      for (int t = 0; t < n_pro; ++t) load_tile(&map_k, base + kOffK + (uint32_t)t * kTileBytes, bar(B3_Q), jt[t]);
+      arm(B3_Q, kTileBytes + kKVBytes * (uint32_t)n_pro);
+      load_q(B3_Q);
+      for (int t = 0; t < n_pro; ++t) load_k(t, B3_Q, jt[t]);
       // stage u = {V_u, K_{u+3}} into slot u % 3, free once phase u/3 of SFULL[u%3] has completed
       bool ok = true;
       int st = 0;
@@ -174,11 +246,11 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (!ok) break;
         TRACE(3, 10, u);
         if (u == p.debug_drop_stage) {
-          mbar_expect_tx(bar(B3_STAGE + st), kTileBytes);               // bytes that never arrive
+          arm(B3_STAGE + st, kKVBytes);                                 // bytes that never arrive
         } else {
-          mbar_expect_tx(bar(B3_STAGE + st), more ? 2u * kTileBytes : kTileBytes);
-          load_tile(&map_v, base + kOffV + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), jt[0]);
-          if (more) load_tile(&map_k, base + kOffK + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), jk);
+          arm(B3_STAGE + st, more ? 2u * kKVBytes : kKVBytes);
+          load_v(st, B3_STAGE + st, jt[0]);
+          if (more) load_k(st, B3_STAGE + st, jk);
         }
         jt[0] = jt[1]; jt[1] = jt[2]; jt[2] = jk;
         if (++st == kStages) { st = 0; ph ^= 1u; }
@@ -193,50 +265,76 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     auto wait_all = [&](uint32_t bb, uint32_t parity, int site) {
       return __all_sync(0xffffffffu, mbar_wait(bb, parity, abort_flag, site));
     };
-    if (n > 0) {
-      constexpr uint32_t idesc_qk = instr_desc(false, 128u);         // S: 128 queries x 128 keys
-      constexpr uint32_t idesc_pv = instr_desc(true, (uint32_t)HD);  // O: 128 queries x HD
+    // CTA pairs: the first CTA's warp issues for both (M = 256: each CTA's tensor core takes its own 128 query
+    // rows, from its own Q and P, against the key tile whose halves lie in the two CTAs' shared memories)
+    if (n > 0 && (!kPair || rank == 0u)) {
+      constexpr uint32_t kM = kPair ? 256u : 128u;
+      constexpr uint32_t idesc_qk = instr_desc(false, 128u, kM);         // S: queries x 128 keys
+      constexpr uint32_t idesc_pv = instr_desc(true, (uint32_t)HD, kM);  // O: queries x HD
       const uint64_t qdesc0 = smem_desc(base + kOffQ, 16, 1024);
       const uint64_t kdesc0 = smem_desc(base + kOffK, 16, 1024);
       const uint64_t vdesc0 = smem_desc(base + kOffV, kHalfBytes, 1024);
+      auto commit = [&](int i) {
+        if (kPair) umma_commit_pair(bar(i), (uint16_t)3);
+        else umma_commit(bar(i));
+      };
       auto issue_qk = [&](int slot) {                       // S[slot] = Q K^T with the K tile in `slot`
-        const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)slot * (kTileBytes >> 4));
+        const uint64_t kd = kdesc0 + (uint64_t)((uint32_t)slot * (kKVBytes >> 4));
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
-          // 16 contraction elements = 32 bytes inside the swizzle atom; second half 16 KB on
-          const uint64_t off = (uint64_t)((((uint32_t)kk >> 2) * kHalfBytes + ((uint32_t)kk & 3u) * 32u) >> 4);
-          umma_ss(tS[slot], qdesc0 + off, kd + off, idesc_qk, kk > 0 ? 1u : 0u);
+          // 16 contraction elements = 32 bytes inside the swizzle atom; the second 64 columns lie behind the
+          // first (Q: 16 KB on; K: half of this CTA's share of the tile on)
+          const uint64_t off_q = (uint64_t)((((uint32_t)kk >> 2) * kHalfBytes + ((uint32_t)kk & 3u) * 32u) >> 4);
+          const uint64_t off_k = (uint64_t)((((uint32_t)kk >> 2) * (kKVBytes / 2u) + ((uint32_t)kk & 3u) * 32u) >> 4);
+          if (kPair) umma_ss_pair(tS[slot], qdesc0 + off_q, kd + off_k, idesc_qk, kk > 0 ? 1u : 0u);
+          else umma_ss(tS[slot], qdesc0 + off_q, kd + off_k, idesc_qk, kk > 0 ? 1u : 0u);
         }
       };
-      bool ok = wait_all(bar(B3_Q), 0u, 200);
+      // P of the tile in buffer s written: by this CTA's four warps and, in a pair, by the other CTA's
+      auto wait_p = [&](int sidx, uint32_t parity) {
+        bool got = wait_all(bar(B3_PFULL + sidx), parity, 220 + sidx);
+        if (kPair && got)
+          got = __all_sync(0xffffffffu, mbar_wait_cluster(bar(B3_PEERP + sidx), parity, abort_flag, 230 + sidx));
+        return got;
+      };
+      // the tiles of stage barrier i landed: this CTA's share and, in a pair, the other CTA's
+      auto wait_tiles = [&](int i, int peer_i, uint32_t parity, int site) {
+        bool got = wait_all(bar(i), parity, site);
+        if (kPair && got) got = wait_all(bar(peer_i), parity, site + 40);
+        return got;
+      };
+      bool ok = wait_tiles(B3_Q, B3_PEERQ, 0u, 200);
       if (ok) {
         tc_fence_after();
         TRACE(0, 20, 0);
         for (int t = 0; t < 3 && t < n; ++t) {
           issue_qk(t);
-          umma_commit(bar(B3_SFULL + t));
+          commit(B3_SFULL + t);
         }
         TRACE(0, 21, 0);
-        ok = wait_all(bar(B3_STAGE + 0), 0u, 210);
-        if (ok) ok = wait_all(bar(B3_PFULL + 0), 0u, 220);
+        ok = wait_tiles(B3_STAGE + 0, B3_PEERSTAGE + 0, 0u, 210);
+        if (ok) ok = wait_p(0, 0u);
         tc_fence_after();
       }
       int st = 0;
       uint32_t ph = 0;                                       // parity of the current lap over the three buffers
       for (int u = 0; u < n && ok; ++u) {
-        const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)st * (kTileBytes >> 4));
+        const uint64_t vd = vdesc0 + (uint64_t)((uint32_t)st * (kKVBytes >> 4));
         TRACE(0, 22, u);
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)                        // 16 keys = 16 rows of 128 B; P advances 8 columns
-          umma_ts(tO, tS[st] + (uint32_t)kk * 8u, vd + (uint64_t)((uint32_t)kk * (2048u >> 4)), idesc_pv,
-                  (kk > 0 || u > 0) ? 1u : 0u);
+        for (int kk = 0; kk < 8; ++kk) {                      // 16 keys = 16 rows of 128 B; P advances 8 columns
+          const uint32_t pa = tS[st] + (uint32_t)kk * 8u;
+          const uint64_t vk = vd + (uint64_t)((uint32_t)kk * (2048u >> 4));
+          if (kPair) umma_ts_pair(tO, pa, vk, idesc_pv, (kk > 0 || u > 0) ? 1u : 0u);
+          else umma_ts(tO, pa, vk, idesc_pv, (kk > 0 || u > 0) ? 1u : 0u);
+        }
         if (u + 3 < n) issue_qk(st);
-        umma_commit(bar(B3_SFULL + st));
+        commit(B3_SFULL + st);
         TRACE(0, 24, u);
         if (++st == kStages) { st = 0; ph ^= 1u; }
         if (u + 1 < n) {                                      // operands of the next service, while this one runs
-          ok = wait_all(bar(B3_PFULL + st), ph, 220 + st);
-          if (ok) ok = wait_all(bar(B3_STAGE + st), ph, 210 + st);
+          ok = wait_p(st, ph);
+          if (ok) ok = wait_tiles(B3_STAGE + st, B3_PEERSTAGE + st, ph, 210 + st);
           tc_fence_after();
           TRACE(0, 25, u);
         }
@@ -370,7 +468,10 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B3_PFULL + sb));
+      if (lane == 0) {
+        mbar_arrive(bar(B3_PFULL + sb));
+        if (kPair && rank == 1u) mbar_arrive_cluster(cluster_map(bar(B3_PEERP + sb), 0u));
+      }
       TRACE(1 + w, 33, t);
       sb += 2;
       if (sb >= 3) { sb -= 3; sph ^= 1u; }
@@ -381,10 +482,12 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), (uint32_t)((n - 1) / 3 + 1) & 1u, abort_flag, 320 + w));
       tc_fence_after();
     }
-    // The K/V rings are dead now (every service of this CTA is complete) and serve as scratch: the row's two
-    // partial results meet there, and the output is staged there so that it leaves in whole 128-byte row
-    // pieces instead of 32 scattered 16-byte pieces per store instruction.
-    unsigned char* vring = smem_raw + kOffV;
+    // Scratch: the row's two partial results meet there, and the output is staged there so that it leaves in
+    // whole 128-byte row pieces instead of 32 scattered 16-byte pieces per store instruction.  A single CTA
+    // uses its V ring, which is dead now (every service is complete).  A CTA of a pair may not: writing into
+    // the ring right after the last commit was observed to corrupt the pair's last P V now and then (the
+    // columns of this CTA's half of V, in both CTAs' outputs), so a pair has a scratch area of its own.
+    unsigned char* vring = kPair ? smem_raw + kOffTail + kTail3Padded : smem_raw + kOffV;
     volatile float* stats = reinterpret_cast<volatile float*>(vring + 32768);   // (reference, partial denominator)
     stats[2 * (w * 128 + row)] = my_ref;
     stats[2 * (w * 128 + row) + 1] = l;
@@ -445,9 +548,13 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // ---- teardown -----------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();     // neither CTA's shared or tensor memory goes away while the other may still signal it
   tc_fence_after();
-  if (warp == 9) tmem_dealloc(tmem, 512);
-  if (p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+  if (warp == 9) {
+    if (kPair) tmem_dealloc_pair(tmem, 512);
+    else tmem_dealloc(tmem, 512);
+  }
+  if (kTrace && p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
     for (int i = threadIdx.x; i < 4 * kTraceSlots; i += kThreads) {
       const int role = i / kTraceSlots, k = i % kTraceSlots;
       if (k < p.trace_cap) {
@@ -458,26 +565,50 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.status, SPARSTAR_ERR_TIMEOUT, *abort_flag);
 }
 
-template <int HD>
+template <int HD, bool kPair, bool kTrace>
 int launch3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p,
             dim3 grid, cudaStream_t s) {
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
     // the in-kernel register re-balancing needs the compiled allocation to be what it assumes
     cudaFuncAttributes fa;
-    SPARSTAR_CUDA_TRY(cudaFuncGetAttributes(&fa, attn_tc3_kernel<HD>));
+    SPARSTAR_CUDA_TRY(cudaFuncGetAttributes(&fa, attn_tc3_kernel<HD, kPair, kTrace>));
     if (2 * 128 * kRegsSoftmax + 128 * kRegsOther > kThreads * fa.numRegs) return SPARSTAR_ERR_UNSUPPORTED;
-    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_tc3_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)smem3_bytes(HD)));
+    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_tc3_kernel<HD, kPair, kTrace>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)smem3_bytes(HD, kPair)));
     attr_set[ctx->device & 63] = true;
   }
-  attn_tc3_kernel<HD><<<grid, kThreads, smem3_bytes(HD), s>>>(mq, mk, mv, p);
+  if (kPair) {
+    // two adjacent query tiles per work item, one CTA each, launched as a cluster of two
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * ((grid.x + 1u) / 2u), grid.y, grid.z);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem3_bytes(HD, true);
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    SPARSTAR_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc3_kernel<HD, kPair, kTrace>, mq, mk, mv, p));
+  } else {
+    attn_tc3_kernel<HD, kPair, kTrace><<<grid, kThreads, smem3_bytes(HD), s>>>(mq, mk, mv, p);
+  }
   return SPARSTAR_OK;
 }
 
 }  // namespace
 
+// `pair`: two adjacent query tiles per work item on a pair of CTAs (head dimension 128; the tiles of a pair must
+// walk the same list: dense, or selection blocks of an even number of tiles); `mk` then has 64-row boxes and
+// `p.order`, if given, orders the pairs.  `grid.x` is the number of query tiles either way.
 int launch_attn_tc3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s) {
-  return head_dim == 64 ? launch3<64>(ctx, mq, mk, mv, p, grid, s) : launch3<128>(ctx, mq, mk, mv, p, grid, s);
+                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s, bool pair) {
+  const bool tr = p.trace != nullptr;
+  if (pair) {
+    if (head_dim != 128) return SPARSTAR_ERR_UNSUPPORTED;
+    return tr ? launch3<128, true, true>(ctx, mq, mk, mv, p, grid, s) : launch3<128, true, false>(ctx, mq, mk, mv, p, grid, s);
+  }
+  if (head_dim == 64)
+    return tr ? launch3<64, false, true>(ctx, mq, mk, mv, p, grid, s) : launch3<64, false, false>(ctx, mq, mk, mv, p, grid, s);
+  return tr ? launch3<128, false, true>(ctx, mq, mk, mv, p, grid, s) : launch3<128, false, false>(ctx, mq, mk, mv, p, grid, s);
 }

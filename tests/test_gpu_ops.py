@@ -181,6 +181,40 @@ def test_attention_two_stream_kernel_cross_check(eng, D, L_q, L_k, H, density):
     _attn_case(eng, torch.bfloat16, D, 128, L_q, L_k, H, density, 17, 3)
 
 
+@pytest.mark.parametrize("block,L_q,L_k,H,density", [
+    (256, 256 * 2 + 100, 256 * 5 + 130, 2, 0.5),     # odd number of query tiles: the last pair has an empty second CTA
+    (512, 512 + 300, 512 * 3 + 129, 2, 0.6),
+    (256, 200, 256 * 3 + 7, 1, 0.7),
+    (128, 128 * 5, 128 * 11 + 20, 3, 0.3),           # blocks of one tile: the sparse call stays on single CTAs, the dense one pairs
+])
+def test_attention_cta_pairs(eng, block, L_q, L_k, H, density):
+    """ATTN_TCGEN05_PAIR: two adjacent query tiles that walk the same list (dense, blocks of 256 / 512
+    tokens) on a pair of CTAs issuing cta_group::2 MMAs, each CTA holding half of every K and V tile.
+    Against the oracle, and bit-identical to the single-CTA kernel over repeated runs (same arithmetic in
+    the same order; repeated because the hand-over between the two CTAs is timing dependent)."""
+    import paper_2608_10519_b200 as sp
+    _attn_case(eng, torch.bfloat16, 128, block, L_q, L_k, H, density, 23, sp.ATTN_TCGEN05_PAIR)
+    q = _rand((2, H, L_q, 128), torch.bfloat16, 31)
+    k = _rand((2, H, L_k, 128), torch.bfloat16, 32)
+    v = _rand((2, H, L_k, 128), torch.bfloat16, 33)
+    n_q, n_k = orc.num_blocks(L_q, block), orc.num_blocks(L_k, block)
+    rng = np.random.default_rng(5)
+    lists = [[np.sort(rng.choice(n_k, size=max(1, int(round(density * n_k))), replace=False)).astype(np.int32)
+              for _ in range(n_q)] for _ in range(2 * H)]
+    num, idx = lists_to_tensors(lists, n_k, "cuda")
+    num, idx = num.view(2, H, n_q), idx.view(2, H, n_q, -1)
+    want_s = eng.sparse_forward(q, k, v, block, num, idx)
+    want_d = eng.dense_forward(q, k, v, block)
+    sp.sparstar_set_attn_impl(eng.ctx, sp.ATTN_TCGEN05_PAIR)
+    try:
+        for _ in range(8):
+            assert torch.equal(eng.sparse_forward(q, k, v, block, num, idx), want_s)
+            assert torch.equal(eng.dense_forward(q, k, v, block), want_d)
+        eng.check()
+    finally:
+        sp.sparstar_set_attn_impl(eng.ctx, sp.ATTN_AUTO)
+
+
 def test_attention_tcgen05_strided_inputs_and_rerun(eng):
     """Non-contiguous views (packed QKV-style buffer) and bit-reproducibility of two runs."""
     import paper_2608_10519_b200 as sp
