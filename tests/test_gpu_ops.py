@@ -575,6 +575,35 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(eng):
     compare.check_output(f64(o[0, 0]), want, "bf16")
 
 
+def test_bounded_wait_in_a_cta_pair(eng):
+    """The same without a fault for a pair of CTAs: neither producer copies stage 1, the issuing warp's
+    wait runs out in the first CTA, the second CTA's own waits run out beside it, both meet at the
+    cluster barrier, tensor memory is released; the next call in pair mode is healthy."""
+    import time
+    import paper_2608_10519_b200 as sp
+    q = _rand((1, 1, 256, 128), torch.bfloat16, 83)
+    k = _rand((1, 1, 128 * 6, 128), torch.bfloat16, 84)
+    o = torch.empty_like(q)
+    sp.sparstar_set_attn_impl(eng.ctx, sp.ATTN_TCGEN05_PAIR)
+    try:
+        sp.sparstar_set_debug(eng.ctx, True, 1)
+        try:
+            torch.cuda.synchronize()
+            t0 = time.time()
+            sp.sparstar_attn_fwd(eng.ctx, q, k, k, o, 128, 128 ** -0.5)      # one pair, six tiles
+            st, site = sp.sparstar_check(eng.ctx)
+            elapsed = time.time() - t0
+        finally:
+            sp.sparstar_set_debug(eng.ctx, True, -1)
+        assert st == sp.ERR_TIMEOUT and site != 0 and elapsed < 5.0, (st, site, elapsed)
+        sp.sparstar_attn_fwd(eng.ctx, q, k, k, o, 128, 128 ** -0.5)
+        assert sp.sparstar_check(eng.ctx)[0] == sp.OK
+    finally:
+        sp.sparstar_set_attn_impl(eng.ctx, sp.ATTN_AUTO)
+    want, _ = orc.dense_attention(f64(q[0, 0]), f64(k[0, 0]), f64(k[0, 0]), 128 ** -0.5)
+    compare.check_output(f64(o[0, 0]), want, "bf16")
+
+
 @pytest.mark.parametrize("L_q,L_k,H,density", [(128, 128, 1, 1.0), (128 * 2 + 50, 128 * 7 + 3, 2, 0.5), (128 * 3, 128 * 20, 2, 0.2)])
 def test_attention_tcgen05_head_dim_64(eng, L_q, L_k, H, density):
     _attn_case(eng, torch.bfloat16, 64, 128, L_q, L_k, H, density, 19, 2)
