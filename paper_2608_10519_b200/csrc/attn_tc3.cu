@@ -63,8 +63,7 @@ constexpr uint32_t smem3_tiles(int hd, bool pair = false) {
   return (1u + (pair ? 1u : 2u) * kStages) * (128u * (uint32_t)hd * 2u);
 }
 constexpr uint32_t kOff3Misc = 8u * 24u;                         // after the barrier area (24 slots)
-constexpr uint32_t kOff3Lsum = kOff3Misc + 16u;                  // 2 x 128 floats: partial denominators at the final reference
-constexpr uint32_t kOff3Mref = kOff3Lsum + 2u * 128u * 4u;       // 128 floats: the rows' published references
+constexpr uint32_t kOff3Mref = kOff3Misc + 16u;                  // 128 floats: the rows' published references
 constexpr uint32_t kOff3Trace = kOff3Mref + 128u * 4u;
 constexpr uint32_t kTail3Bytes = kOff3Trace + 4u * kTraceSlots * 4u;
 // A CTA of a pair has an epilogue scratch of its own behind the tail (34 KB used); a single CTA reuses its V ring
