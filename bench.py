@@ -479,6 +479,9 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="use only the first HEADS heads (profiling captures)")
     ap.add_argument("--block", type=int, default=0, help="override the workload's selection block size (profiling captures)")
     ap.add_argument("--impl", default="sparstar", choices=["sparstar", "reference"])
+    ap.add_argument("--score-impl", type=int, default=0,
+                    help="scoring path of the library (sparstar_score_impl; 0 = fp64 MMA fused with the selection, "
+                         "1 = tcgen05 split-bf16 pre-score launch + selection with exact re-scoring near the cutoff)")
     ap.add_argument("--attn-impl", type=int, default=0,
                     help="attention implementation of the library (sparstar_attn_impl; 0 = default, 4 = CTA pairs where "
                          "two query tiles share a list: the dense comparison and blocks of 256 / 512 tokens)")
@@ -536,6 +539,8 @@ def main():
     eng = SparstarAttention(local)
     if args.attn_impl:
         sp.sparstar_set_attn_impl(eng.ctx, args.attn_impl)
+    if args.score_impl:
+        sp.sparstar_set_score_impl(eng.ctx, args.score_impl)
     ctx = eng.ctx
     B, H, D, blk = w.B, w.H, w.D, w.block
     scale = D ** -0.5
