@@ -234,6 +234,34 @@ def test_attention_tcgen05_strided_inputs_and_rerun(eng):
         compare.check_output(f64(o1[0, h]), want, "bf16")
 
 
+def test_attention_tcgen05_strided_output(eng):
+    """The output may be a view too (rows of a wider buffer, heads interleaved): the staged row-contiguous stores
+    must land where the strides say and leave the gaps alone."""
+    import paper_2608_10519_b200 as sp
+    L_q, L_k, H = 128 * 2 + 70, 128 * 5 + 9, 2
+    q = _rand((1, H, L_q, 128), torch.bfloat16, 41)
+    k = _rand((1, H, L_k, 128), torch.bfloat16, 42)
+    v = _rand((1, H, L_k, 128), torch.bfloat16, 43)
+    n = orc.num_blocks(L_k, 128)
+    lists = [[np.arange(i % 2, n, 2, dtype=np.int32) for i in range(orc.num_blocks(L_q, 128))] for _ in range(H)]
+    num, idx = lists_to_tensors(lists, n, "cuda")
+    buf = torch.full((1, L_q, H, 192), 3.0, dtype=torch.bfloat16, device="cuda")     # [B, L, H, 192]: 64 spare columns
+    o = buf[..., :128].permute(0, 2, 1, 3)                                            # [1, H, L_q, 128] view
+    sp.sparstar_sparse_attn_fwd(eng.ctx, q, k, v, o, 128, 128 ** -0.5, num, idx)
+    eng.check()
+    assert torch.all(buf[..., 128:] == 3.0)
+    for h in range(H):
+        want, _ = orc.sparse_attention(f64(q[0, h]), f64(k[0, h]), f64(v[0, h]), lists[h], 128, 128 ** -0.5)
+        compare.check_output(f64(o[0, h]), want, "bf16")
+    buf.fill_(3.0)
+    sp.sparstar_attn_fwd(eng.ctx, q, k, v, o, 128, 128 ** -0.5)
+    eng.check()
+    assert torch.all(buf[..., 128:] == 3.0)
+    for h in range(H):
+        want, _ = orc.dense_attention(f64(q[0, h]), f64(k[0, h]), f64(v[0, h]), 128 ** -0.5)
+        compare.check_output(f64(o[0, h]), want, "bf16")
+
+
 def test_tcgen05_bad_list_entry_is_flagged(eng):
     import paper_2608_10519_b200 as sp
     q = _rand((1, 1, 128, 128), torch.bfloat16, 20)
