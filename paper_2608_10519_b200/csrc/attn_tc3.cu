@@ -37,6 +37,14 @@
 // (wait until every earlier P V has landed, scale O in place, publish), and redo the tile's P from
 // the scores (lower half still in registers, upper half still in tensor memory).
 //
+// CTA pairs (template flag; opt-in).  Where two adjacent query tiles walk the same list (dense; selection
+// blocks of 256 / 512 tokens), a cluster of two CTAs serves them: each CTA has the structure above in its
+// own tensor memory, holds its own Q tile and HALF of every K tile (64 keys) and V tile (64 columns), and one
+// thread of the first CTA issues tcgen05.mma.cta_group::2 with M = 256 for both, followed by one commit
+// that arrives on both CTAs' SFULL barriers.  The second CTA's copies and P releases are counted on
+// barriers of the first CTA (PEERQ, PEERSTAGE, PEERP).  It halves the L2 -> shared-memory bytes and is
+// slower than single CTAs (P V of a tile has to wait for both CTAs' softmax), hence not the default.
+//
 // Every wait on an mbarrier is bounded (about a second); on expiry the CTA records
 // SPARSTAR_ERR_TIMEOUT, all roles leave their loops, tensor memory is released and the kernel
 // returns.
@@ -66,12 +74,7 @@ constexpr uint32_t kOff3Misc = 8u * 24u;                         // after the ba
 constexpr uint32_t kOff3Mref = kOff3Misc + 16u;                  // 128 floats: the rows' published references
 constexpr uint32_t kOff3Trace = kOff3Mref + 128u * 4u;
 constexpr uint32_t kTail3Bytes = kOff3Trace + 4u * kTraceSlots * 4u;
-// A CTA of a pair has an epilogue scratch of its own behind the tail (34 KB used); a single CTA reuses its V ring
-constexpr uint32_t kTail3Padded = (kTail3Bytes + 1023u) & ~1023u;
-constexpr uint32_t kPairScratch = 36u * 1024u;
-constexpr uint32_t smem3_bytes(int hd, bool pair = false) {
-  return smem3_tiles(hd, pair) + (pair ? kTail3Padded + kPairScratch : kTail3Bytes);
-}
+constexpr uint32_t smem3_bytes(int hd, bool pair = false) { return smem3_tiles(hd, pair) + kTail3Bytes; }
 static_assert(B3_COUNT <= 24, "barrier area");
 static_assert(smem3_bytes(128) <= 232448u, "shared memory per CTA");
 
@@ -477,16 +480,21 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     // ---- normalise and write O --------------------------------------------------------------
     if (ok && n > 0) {                              // the completion of the last service
+      // = phase (n-1)/3 + 1 of the last tile's barrier.  A parity wait is only right for a thread that is at most
+      // one phase behind: the warpgroup that owns the last tile has consumed phase (n-1)/3 ("its scores are
+      // ready"), the other one has not and must pass it first - otherwise, arriving while that phase is still
+      // open, it would take the phase before it (same parity as the one it wants) for the end of the kernel.
       const int lb = (n - 1) % 3;
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), (uint32_t)((n - 1) / 3 + 1) & 1u, abort_flag, 320 + w));
+      const uint32_t kph = (uint32_t)((n - 1) / 3);
+      if (((n - 1) & 1) != w)
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), kph & 1u, abort_flag, 325 + w));
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + lb), (kph + 1u) & 1u, abort_flag, 320 + w));
       tc_fence_after();
     }
-    // Scratch: the row's two partial results meet there, and the output is staged there so that it leaves in
-    // whole 128-byte row pieces instead of 32 scattered 16-byte pieces per store instruction.  A single CTA
-    // uses its V ring, which is dead now (every service is complete).  A CTA of a pair may not: writing into
-    // the ring right after the last commit was observed to corrupt the pair's last P V now and then (the
-    // columns of this CTA's half of V, in both CTAs' outputs), so a pair has a scratch area of its own.
-    unsigned char* vring = kPair ? smem_raw + kOffTail + kTail3Padded : smem_raw + kOffV;
+    // The V ring is dead now (every service is complete) and serves as scratch: the row's two partial results
+    // meet there, and the output is staged there so that it leaves in whole 128-byte row pieces instead of 32
+    // scattered 16-byte pieces per store instruction.
+    unsigned char* vring = smem_raw + kOffV;
     volatile float* stats = reinterpret_cast<volatile float*>(vring + 32768);   // (reference, partial denominator)
     stats[2 * (w * 128 + row)] = my_ref;
     stats[2 * (w * 128 + row) + 1] = l;
