@@ -63,9 +63,10 @@ typedef enum {
   SPARSTAR_ATTN_AUTO = 0,        /* tensor-core kernel when the shape allows, else SIMT */
   SPARSTAR_ATTN_SIMT = 1,        /* fp32 FFMA kernel (any supported shape) */
   SPARSTAR_ATTN_TCGEN05 = 2,     /* tcgen05/TMEM/TMA kernels (bf16, D in {64,128}, block in {32,64,128,256,512});
-                                    blocks >= 128 and dense: three score tiles in flight, one accumulator */
-  SPARSTAR_ATTN_TCGEN05_2STREAM = 3, /* same shapes; blocks >= 128 and dense on the older two-stream kernel (two
-                                    score tiles, two accumulators merged at the end) - kept as a cross-check */
+                                    three score tiles in flight, one accumulator; blocks of 64 / 32 tokens are
+                                    gathered two / four to a 128-key tile */
+  SPARSTAR_ATTN_TCGEN05_2STREAM = 3, /* same shapes on the older two-stream kernel (two score tiles, two accumulators
+                                    merged at the end) - kept as a cross-check */
   SPARSTAR_ATTN_TCGEN05_PAIR = 4  /* same shapes; where two adjacent 128-row query tiles walk the same list (dense,
                                     blocks of 256 or 512 tokens) and D = 128, they run on a pair of CTAs that issue
                                     tcgen05.mma.cta_group::2 together, each holding half of every K and V tile;

@@ -1,3 +1,5 @@
+// The older two-stream form of the attention kernel, kept as a cross-check of the three-tile kernel
+// (attn_tc3.cu) and as the block-mass kernel, and the launcher of both.
 // Block-sparse / dense attention forward for bf16 on the sm_100a tensor cores (Eq. 7: softmax
 // over the keys of the retained blocks A_i, tiles outside A_i skipped).  Head dimension 128 or
 // 64; selection blocks of 128, 256 or 512 tokens, always walked as tiles of 128 tokens, or of 64 /
@@ -766,8 +768,10 @@ int launch_attn_tc(sparstar_ctx* ctx, const AttnArgs& a, cudaStream_t s) {
   p.debug_drop_stage = ctx->debug_drop_stage;
   dim3 grid(p.n_q, a.q.H, a.q.B);
   int st2;
-  if (gather > 1)
+  if (gather > 1 && ctx->attn_impl == SPARSTAR_ATTN_TCGEN05_2STREAM)
     st2 = a.q.D == 64 ? launch_variant<2, 64>(ctx, mq, mk, mv, p, grid, s) : launch_variant<2, 128>(ctx, mq, mk, mv, p, grid, s);
+  else if (gather > 1)
+    st2 = launch_attn_tc3(ctx, mq, mk, mv, p, a.q.D, grid, s, false, true);
   else if (ctx->attn_impl == SPARSTAR_ATTN_TCGEN05_2STREAM)
     st2 = a.q.D == 64 ? launch_variant<0, 64>(ctx, mq, mk, mv, p, grid, s) : launch_variant<0, 128>(ctx, mq, mk, mv, p, grid, s);
   else

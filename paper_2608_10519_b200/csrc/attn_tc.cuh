@@ -127,4 +127,4 @@ int make_map(CUtensorMap* map, const sparstar_tensor& t, int box_rows = 128) {
 // The three-tile pipeline (attn_tc3.cu): same parameters, lists of whole 128-token tiles or
 // selection blocks that are multiples of a tile (p.gather == 1), attention only.
 int launch_attn_tc3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s, bool pair = false);
+                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s, bool pair = false, bool gathered = false);

@@ -1,6 +1,8 @@
 // Block-sparse / dense attention forward for bf16 on the sm_100a tensor cores, three-tile pipeline
 // (Eq. 7: softmax over the keys of the retained blocks A_i, tiles outside A_i skipped).  Head
-// dimension 128 or 64; selection blocks of 128, 256 or 512 tokens walked as tiles of 128 tokens.
+// dimension 128 or 64; selection blocks of 128, 256 or 512 tokens walked as tiles of 128 tokens, or of 64 /
+// 32 tokens (template flag: the query blocks of a tile share the union of their lists, two / four listed key
+// blocks are gathered into one tile, each row masks what its own query block does not keep).
 //
 // One CTA per (batch, head, 128-row query tile).  Tensor memory holds THREE score tiles and ONE
 // output accumulator (S0 | S1 | S2 | O): tile t of the key-block list lives in score buffer t % 3
@@ -78,12 +80,13 @@ constexpr uint32_t smem3_bytes(int hd, bool pair = false) { return smem3_tiles(h
 static_assert(B3_COUNT <= 24, "barrier area");
 static_assert(smem3_bytes(128) <= 232448u, "shared memory per CTA");
 
-template <int HD, bool kPair, bool kTrace>
+template <int HD, bool kPair, bool kTrace, bool kGather>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, const TcParams p) {
   static_assert(HD == 64 || HD == 128, "head dimension");
   static_assert(!kPair || HD == 128, "CTA pairs: head dimension 128");
+  static_assert(!(kPair && kGather), "gathered blocks run on single CTAs");
   constexpr uint32_t kTileBytes = 128u * HD * 2u;
   constexpr uint32_t kKVBytes = kPair ? kTileBytes / 2u : kTileBytes;   // this CTA's share of a K or V tile
   constexpr uint32_t kOffK = kOffQ + kTileBytes;
@@ -125,8 +128,13 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   const int* list = dense ? nullptr : p.kv_indices + row_id * (size_t)p.cap;
   const int cnt = dense ? 0 : max(min(p.kv_num_blocks[row_id], p.cap), 0);
   // tiles to walk: every listed block contributes m tiles, except that the last key block may hold fewer
-  int n = dense ? p.n_k : cnt * p.m;
-  if (!dense && p.m > 1 && cnt > 0 && list[cnt - 1] == p.n_kb - 1) n -= p.m * p.n_kb - p.n_k;
+  // kGather: selection blocks shorter than a tile.  The list then belongs to the query TILE (the union of its
+  // query blocks' lists, entries (block << 4) | bits, bit s = kept by the tile's s-th query block) and
+  // p.gather listed blocks are gathered into each 128-key tile; a row masks what its own block does not keep.
+  const int gather = kGather ? p.gather : 1;
+  const int sub_rows = kBlock / gather;           // tokens of a gathered block
+  int n = dense ? p.n_k : (kGather ? (cnt + gather - 1) / gather : cnt * p.m);
+  if (!kGather && !dense && p.m > 1 && cnt > 0 && list[cnt - 1] == p.n_kb - 1) n -= p.m * p.n_kb - p.n_k;
   const int q_row0 = qi * kBlock;
 
   if (threadIdx.x == 0) {
@@ -167,7 +175,53 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   if (warp == 8) {
     // ================================ TMA producer ======================================
     reg_dec<kRegsOther>();
-    if (lane == 0 && n > 0) {
+    if (kGather) {
+      // Lane s < gather owns the tile's s-th listed block: it reads the entry and issues that block's copies, so a
+      // tile's 4 * gather copies leave as four instructions; lane 0 also arms the barriers, copies Q and waits.
+      if (n > 0) {
+        const bool active = lane < gather;
+        auto my_row = [&](int t) {                     // a missing entry repeats the tile's first
+          int e = t * gather + lane;
+          if (!active || e >= cnt) e = t * gather;
+          return min(max(list[e] >> 4, 0), p.n_kb - 1) * sub_rows;
+        };
+        auto load_part = [&](const CUtensorMap* map, uint32_t dst, uint32_t barrier, int r) {
+          const uint32_t d = dst + (uint32_t)(lane * sub_rows) * 128u;     // 128-byte rows inside a column half
+          tma_load_4d(d, map, barrier, 0, r, h, b);
+          if (HD == 128) tma_load_4d(d + kHalfBytes, map, barrier, 64, r, h, b);
+        };
+        int rt[3] = {0, 0, 0};
+        const int n_pro = min(n, 3);
+        for (int t = 0; t < n_pro; ++t) rt[t] = my_row(t);
+        if (lane == 0) {
+          mbar_expect_tx(bar(B3_Q), kTileBytes * (uint32_t)(1 + n_pro));
+          tma_load_4d(base + kOffQ, &map_q, bar(B3_Q), 0, q_row0, h, b);
+          if (HD == 128) tma_load_4d(base + kOffQ + kHalfBytes, &map_q, bar(B3_Q), 64, q_row0, h, b);
+        }
+        __syncwarp();
+        if (active)
+          for (int t = 0; t < n_pro; ++t) load_part(&map_k, base + kOffK + (uint32_t)t * kTileBytes, bar(B3_Q), rt[t]);
+        bool ok = true;
+        int st = 0;
+        uint32_t ph = 0;
+        for (int u = 0; u < n && ok; ++u) {
+          const bool more = u + 3 < n;
+          const int rk = more ? my_row(u + 3) : 0;
+          int okk = 1;
+          if (lane == 0) okk = mbar_wait(bar(B3_SFULL + st), ph, abort_flag, 100 + st) ? 1 : 0;
+          ok = __shfl_sync(0xffffffffu, okk, 0) != 0;
+          if (!ok) break;
+          if (lane == 0) mbar_expect_tx(bar(B3_STAGE + st), more ? 2u * kTileBytes : kTileBytes);
+          __syncwarp();
+          if (active) {
+            load_part(&map_v, base + kOffV + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), rt[0]);
+            if (more) load_part(&map_k, base + kOffK + (uint32_t)st * kTileBytes, bar(B3_STAGE + st), rk);
+          }
+          rt[0] = rt[1]; rt[1] = rt[2]; rt[2] = rk;
+          if (++st == kStages) { st = 0; ph ^= 1u; }
+        }
+      }
+    } else if (lane == 0 && n > 0) {
       int prev = -1;
       auto checked = [&](int j, bool first_of_block) {
         if (j < 0 || j >= p.n_kb || (first_of_block && j <= prev)) {   // malformed: flag it, stay in bounds
@@ -353,19 +407,61 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const float c = p.scale * 1.4426950408889634f;  // logits in log2 units
     // valid key columns of the last tile: lists ascend, so only the final entry can be the partial last key block
     int last_valid = kBlock;
-    if (n > 0 && (dense || list[cnt - 1] == p.n_kb - 1)) last_valid = p.L_k - (p.n_k - 1) * kBlock;
+    if (!kGather && n > 0 && (dense || list[cnt - 1] == p.n_kb - 1)) last_valid = p.L_k - (p.n_k - 1) * kBlock;
+    const int row_group = row / sub_rows;           // gathered blocks: which of the tile's query blocks owns this row
+    const int tail_sub = p.L_k - (p.n_kb - 1) * sub_rows;     // keys of the last (possibly partial) gathered block
     float my_ref = -INFINITY;                       // the reference my P and partial denominator are expressed in
     float l = 0.f;
     bool ok = true;
     int sb = w;                                     // t % 3
     uint32_t sph = 0;                               // (t / 3) & 1
     for (int t = w; t < n && ok; t += 2) {
+      // gathered blocks: this tile's union entries, fetched before the wait so that the loads are not on the
+      // critical path (0 = no entry)
+      int ent[4] = {0, 0, 0, 0};
+      if (kGather) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int e = t * gather + g;
+          if (g < gather && e < cnt) ent[g] = list[e];
+        }
+      }
       ok = __all_sync(0xffffffffu, mbar_wait(bar(B3_SFULL + sb), sph, abort_flag, 300 + w));
       if (!ok) break;
       tc_fence_after();
       TRACE(1 + w, 30, t);
-      int c0 = 32, c1 = 32, c2 = 32, c3 = 32;       // valid columns of the tile's four 32-column segments
-      if (t == n - 1 && last_valid < kBlock) {
+      // Valid columns of the tile's four 32-column segments for this row.  Gathered blocks: an entry counts only
+      // if this row's query block keeps it (rows of one warp share a query block, so all of this is warp-uniform).
+      int c0 = 32, c1 = 32, c2 = 32, c3 = 32;
+      if (kGather) {
+        int vc[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          vc[g] = 0;
+          if ((ent[g] >> row_group) & 1) vc[g] = (ent[g] >> 4) == p.n_kb - 1 ? tail_sub : sub_rows;
+        }
+        if (gather == 4) {
+          c0 = vc[0]; c1 = vc[1]; c2 = vc[2]; c3 = vc[3];
+        } else {
+          c0 = min(vc[0], 32); c1 = max(vc[0] - 32, 0); c2 = min(vc[1], 32); c3 = max(vc[1] - 32, 0);
+        }
+        if ((c0 | c1 | c2 | c3) == 0) {
+          // nothing of this tile is kept by the row's query block: P = 0, no exponentials, the reference and the
+          // denominator stay as they are (a later tile adopts whatever has been published meanwhile)
+          uint32_t zero[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) zero[i] = 0u;
+          tmem_st32(tS[sb] + lane_off, zero);
+          tmem_st32(tS[sb] + lane_off + 32u, zero);
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(B3_PFULL + sb));
+          sb += 2;
+          if (sb >= 3) { sb -= 3; sph ^= 1u; }
+          continue;
+        }
+      } else if (t == n - 1 && last_valid < kBlock) {
         c0 = min(max(last_valid, 0), 32); c1 = min(max(last_valid - 32, 0), 32);
         c2 = min(max(last_valid - 64, 0), 32); c3 = min(max(last_valid - 96, 0), 32);
       }
@@ -572,16 +668,16 @@ attn_tc3_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   if (threadIdx.x == 0 && *abort_flag != 0) record_status(p.status, SPARSTAR_ERR_TIMEOUT, *abort_flag);
 }
 
-template <int HD, bool kPair, bool kTrace>
+template <int HD, bool kPair, bool kTrace, bool kGather>
 int launch3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& p,
             dim3 grid, cudaStream_t s) {
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
     // the in-kernel register re-balancing needs the compiled allocation to be what it assumes
     cudaFuncAttributes fa;
-    SPARSTAR_CUDA_TRY(cudaFuncGetAttributes(&fa, attn_tc3_kernel<HD, kPair, kTrace>));
+    SPARSTAR_CUDA_TRY(cudaFuncGetAttributes(&fa, attn_tc3_kernel<HD, kPair, kTrace, kGather>));
     if (2 * 128 * kRegsSoftmax + 128 * kRegsOther > kThreads * fa.numRegs) return SPARSTAR_ERR_UNSUPPORTED;
-    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_tc3_kernel<HD, kPair, kTrace>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    SPARSTAR_CUDA_TRY(cudaFuncSetAttribute(attn_tc3_kernel<HD, kPair, kTrace, kGather>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)smem3_bytes(HD, kPair)));
     attr_set[ctx->device & 63] = true;
   }
@@ -596,9 +692,9 @@ int launch3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, con
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    SPARSTAR_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc3_kernel<HD, kPair, kTrace>, mq, mk, mv, p));
+    SPARSTAR_CUDA_TRY(cudaLaunchKernelEx(&cfg, attn_tc3_kernel<HD, kPair, kTrace, kGather>, mq, mk, mv, p));
   } else {
-    attn_tc3_kernel<HD, kPair, kTrace><<<grid, kThreads, smem3_bytes(HD), s>>>(mq, mk, mv, p);
+    attn_tc3_kernel<HD, kPair, kTrace, kGather><<<grid, kThreads, smem3_bytes(HD), s>>>(mq, mk, mv, p);
   }
   return SPARSTAR_OK;
 }
@@ -607,15 +703,23 @@ int launch3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, con
 
 // `pair`: two adjacent query tiles per work item on a pair of CTAs (head dimension 128; the tiles of a pair must
 // walk the same list: dense, or selection blocks of an even number of tiles); `mk` then has 64-row boxes and
-// `p.order`, if given, orders the pairs.  `grid.x` is the number of query tiles either way.
+// `p.order`, if given, orders the pairs.  `gathered`: selection blocks of 64 / 32 tokens (p.gather = 2 / 4, union
+// lists per query tile, K/V maps with boxes of that many rows).  `grid.x` is the number of query tiles either way.
 int launch_attn_tc3(sparstar_ctx* ctx, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s, bool pair) {
+                    const TcParams& p, int head_dim, dim3 grid, cudaStream_t s, bool pair, bool gathered) {
   const bool tr = p.trace != nullptr;
   if (pair) {
-    if (head_dim != 128) return SPARSTAR_ERR_UNSUPPORTED;
-    return tr ? launch3<128, true, true>(ctx, mq, mk, mv, p, grid, s) : launch3<128, true, false>(ctx, mq, mk, mv, p, grid, s);
+    if (head_dim != 128 || gathered) return SPARSTAR_ERR_UNSUPPORTED;
+    return tr ? launch3<128, true, true, false>(ctx, mq, mk, mv, p, grid, s)
+              : launch3<128, true, false, false>(ctx, mq, mk, mv, p, grid, s);
+  }
+  if (gathered) {
+    if (head_dim == 64) return launch3<64, false, false, true>(ctx, mq, mk, mv, p, grid, s);
+    return launch3<128, false, false, true>(ctx, mq, mk, mv, p, grid, s);
   }
   if (head_dim == 64)
-    return tr ? launch3<64, false, true>(ctx, mq, mk, mv, p, grid, s) : launch3<64, false, false>(ctx, mq, mk, mv, p, grid, s);
-  return tr ? launch3<128, false, true>(ctx, mq, mk, mv, p, grid, s) : launch3<128, false, false>(ctx, mq, mk, mv, p, grid, s);
+    return tr ? launch3<64, false, true, false>(ctx, mq, mk, mv, p, grid, s)
+              : launch3<64, false, false, false>(ctx, mq, mk, mv, p, grid, s);
+  return tr ? launch3<128, false, true, false>(ctx, mq, mk, mv, p, grid, s)
+            : launch3<128, false, false, false>(ctx, mq, mk, mv, p, grid, s);
 }

@@ -473,21 +473,24 @@ def test_trace_records_role_events(eng):
 @pytest.mark.parametrize("D", [128, 64])
 @pytest.mark.parametrize("L_q,L_k,density", [(64 * 5 + 20, 64 * 31 + 9, 0.3), (64, 64, 1.0), (50, 64 * 3 + 1, 1.0),
                                              (64 * 3, 64 * 20, 0.05), (64 * 2 + 1, 64 * 9 + 63, 0.5)])
-def test_attention_tcgen05_block64(eng, D, L_q, L_k, density):
-    """Selection blocks of 64 tokens on the tensor-core kernel: two listed blocks are gathered
+@pytest.mark.parametrize("impl", [2, 3])
+def test_attention_tcgen05_block64(eng, D, L_q, L_k, density, impl):
+    """Selection blocks of 64 tokens on the tensor-core kernels (impl 2: the three-tile kernel's gathered
+    instance; impl 3: the older two-stream kernel's, as a cross-check): two listed blocks are gathered
     into one 128-key tile (odd list lengths leave half a tile unused, the last block may be
-    partial) and a CTA's query tile holds one 64-row query block."""
-    _attn_case(eng, torch.bfloat16, D, 64, L_q, L_k, 2, density, 23, 2)
+    partial) and a CTA's query tile holds two 64-row query blocks."""
+    _attn_case(eng, torch.bfloat16, D, 64, L_q, L_k, 2, density, 23, impl)
 
 
 @pytest.mark.parametrize("D", [128, 64])
 @pytest.mark.parametrize("L_q,L_k,density", [(32 * 5 + 20, 32 * 61 + 9, 0.3), (32, 32, 1.0), (20, 32 * 3 + 1, 1.0),
                                              (32 * 3, 32 * 40, 0.05), (32 * 2 + 1, 32 * 18 + 31, 0.5),
                                              (32 * 2, 32 * 7, 0.72), (32 * 2, 32 * 6, 0.99)])
-def test_attention_tcgen05_block32(eng, D, L_q, L_k, density):
+@pytest.mark.parametrize("impl", [2, 3])
+def test_attention_tcgen05_block32(eng, D, L_q, L_k, density, impl):
     """Selection blocks of 32 tokens: four listed blocks per 128-key tile, list lengths of every
-    residue modulo four, a partial last block."""
-    _attn_case(eng, torch.bfloat16, D, 32, L_q, L_k, 2, density, 29, 2)
+    residue modulo four, a partial last block (both tensor-core kernels, as above)."""
+    _attn_case(eng, torch.bfloat16, D, 32, L_q, L_k, 2, density, 29, impl)
 
 
 @pytest.mark.parametrize("block,L_q,L_k", [(256, 256 * 2 + 100, 256 * 5 + 130), (256, 200, 256 * 3 + 7), (512, 512 + 300, 512 * 3 + 129)])
